@@ -1,0 +1,154 @@
+/*
+ * rmm.h - C ABI of the randomized-matrix-multiplication (RMM) linear layer for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The layer is the one of "Memory-Efficient Backpropagation through Large Linear
+ * Layers" (arXiv 2201.13195), Section 2.1, Algorithm 1: the forward pass returns
+ * Y = X W^T + 1 b^T (Eq. 1) and keeps, instead of X, the sketch X_proj = S^T X
+ * together with the seed that S was drawn from; the backward pass regenerates S,
+ * and returns the exact dX = dY W (Eq. 2), the randomized estimate
+ * dW = (dY^T S) X_proj of dY^T X (Eq. 4) and the exact db = dY^T 1 (Eq. 3).
+ *
+ * Notation: N = number of token rows (the paper's batch dimension B), D_in / D_out =
+ * the paper's N_in / N_out, B_proj = number of columns of S (Section 2.4.2).
+ *
+ * General conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, row-major,
+ *     contiguous, 16-byte aligned.  The library allocates no device memory, keeps no
+ *     state between calls, never synchronises, and enqueues work only on the CUDA
+ *     stream that is passed in (a cudaStream_t cast to void*, NULL = default stream).
+ *   - Outputs are overwritten, never accumulated into.
+ *   - dtype RMM_DTYPE_BF16: tensors are bfloat16, contractions run on the tensor
+ *     cores with fp32 accumulation; D_in and D_out must be multiples of 8.
+ *     dtype RMM_DTYPE_F32: tensors are fp32, contractions are plain fp32 FMA.
+ *   - Errors are return codes.  Argument errors are detected on the host before any
+ *     launch.  A device-side wait that does not complete within its iteration limit
+ *     is recorded in the workspace and reported by rmm_last_device_status().
+ *   - There is no CPU fallback: on a machine without a usable sm_100a device every
+ *     compute entry point returns RMM_ERR_CUDA.
+ *
+ * The sketch matrix S (N x B_proj) is a pure function of (seed, dist, N-index,
+ * column index, dtype); it does not depend on tile shapes, launch geometry or on
+ * which pass asks for it.  S = c * P with c = fp32 1/sqrt(B_proj) and
+ *   RMM_DIST_GAUSSIAN   P iid standard normal (Eq. 5): Philox4x32-10 with key =
+ *                       (seed low word, seed high word) and counter
+ *                       (n >> 3, j, 0, 0) gives four words; word i gives, by a
+ *                       Box-Muller transform on its two 16-bit halves evaluated with
+ *                       a fixed sequence of correctly rounded fp32 operations, the
+ *                       entries P[8*(n>>3) + 2i][j] and P[8*(n>>3) + 2i + 1][j];
+ *   RMM_DIST_RADEMACHER P = +-1 with probability 1/2 (Section 3.2): counter
+ *                       (n >> 7, j, 0, 1) gives 128 bits, entry P[n][j] is -1 when
+ *                       bit (n & 31) of word ((n & 127) >> 5) is set;
+ *   RMM_DIST_IDENTITY   S = I (needs B_proj == N; c = 1): the case in which the
+ *                       layer reduces to the exact linear layer; meant for tests.
+ * In bf16 mode P is rounded to bfloat16 (nearest even) before it is used.
+ */
+#ifndef RMM_H_
+#define RMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RMM_OK = 0,
+  RMM_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, B_proj outside [1,N], bad enum, misalignment */
+  RMM_ERR_UNSUPPORTED = 2, /* shape not supported in this dtype (D_in or D_out not a multiple of 8 in bf16) */
+  RMM_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or smaller than rmm_workspace_bytes() */
+  RMM_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed (including: no sm_100a device) */
+  RMM_ERR_TIMEOUT = 5      /* a device-side wait gave up; results of that call are invalid */
+} rmm_status;
+
+typedef enum { RMM_DIST_GAUSSIAN = 0, RMM_DIST_RADEMACHER = 1, RMM_DIST_IDENTITY = 2 } rmm_dist;
+typedef enum { RMM_DTYPE_BF16 = 0, RMM_DTYPE_F32 = 1 } rmm_dtype;
+
+/*
+ * Bytes of scratch device memory that rmm_forward / rmm_backward need for these
+ * sizes (the larger of the two).  The scratch holds the intermediate G = S^T dY
+ * (B_proj x D_out), partial sums, and a status word.  Returns 0 for invalid sizes.
+ * The same workspace may be reused by later calls on the same stream; calls that may
+ * overlap on the device need separate workspaces.
+ */
+size_t rmm_workspace_bytes(int64_t N, int64_t D_in, int64_t D_out, int64_t B_proj, rmm_dtype dt);
+
+/*
+ * Algorithm 1, FORWARD (Eq. 1 and X_proj = S^T X, Section 2.1).
+ *   in : X [N, D_in], W [D_out, D_in], b [D_out] or NULL (no bias)
+ *   out: Y [N, D_out] = X W^T + 1 b^T ;  X_proj [B_proj, D_in] = S^T X
+ * X_proj and seed are all the caller has to keep for the backward pass.  Use a fresh
+ * seed for every layer and every step: S must be independent of dY (Section 2.1).
+ * Y may be NULL (only the sketch is computed).
+ */
+rmm_status rmm_forward(const void* X, const void* W, const void* b,
+                       int64_t N, int64_t D_in, int64_t D_out,
+                       uint64_t seed, int64_t B_proj, rmm_dist dist, rmm_dtype dt,
+                       void* Y, void* X_proj,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Algorithm 1, BACKWARD (Eq. 2, 3, 4).  (seed, B_proj, dist, N) must be the values
+ * given to the forward call that produced X_proj.
+ *   in : dY [N, D_out], W [D_out, D_in], X_proj [B_proj, D_in]
+ *   out: dX [N, D_in] = dY W               (exact; NULL to skip)
+ *        dW [D_out, D_in] = (S^T dY)^T X_proj   (unbiased estimate of dY^T X)
+ *        db [D_out] = sum over rows of dY  (exact; NULL to skip)
+ * The bias is not an input: Algorithm 1 lists it but no gradient depends on it.
+ */
+rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj,
+                        int64_t N, int64_t D_in, int64_t D_out,
+                        uint64_t seed, int64_t B_proj, rmm_dist dist, rmm_dtype dt,
+                        void* dX, void* dW, void* db,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Writes the sketch matrix itself, S_out [N, B_proj] row-major in the given dtype
+ * holding the UNSCALED entries P (multiply by fp32 1/sqrt(B_proj) to get S, Eq. 5).
+ * Not part of the layer: it exists so that the generator can be compared bit for bit
+ * with an independent implementation.
+ */
+rmm_status rmm_debug_generate_s(uint64_t seed, int64_t N, int64_t B_proj, rmm_dist dist, rmm_dtype dt,
+                                void* S_out, void* cuda_stream);
+
+/*
+ * Reads the status word that the kernels of the last call using this workspace left
+ * there.  HOST-synchronous on the device-to-host copy of one word: the caller must
+ * have synchronised the stream first.  Returns RMM_OK or RMM_ERR_TIMEOUT (or
+ * RMM_ERR_CUDA if the copy fails).
+ */
+rmm_status rmm_last_device_status(const void* workspace);
+
+/* Static, human-readable name of a status code. */
+const char* rmm_status_string(rmm_status s);
+
+/*
+ * Host-buffer convenience wrappers (end-to-end path): the tensor arguments are HOST
+ * pointers (pinned memory recommended); the device buffers dev_* and the workspace
+ * are caller-owned DEVICE scratch of at least the tensors' sizes.  Each call copies
+ * its inputs host->device, runs the device entry point above, and copies the outputs
+ * device->host, all on cuda_stream, then synchronises that stream.
+ *   rmm_forward_host : dev_in  >= bytes(X) + bytes(W) + bytes(b), dev_out >= bytes(Y) + bytes(X_proj)
+ *   rmm_backward_host: dev_in  >= bytes(dY) + bytes(W) + bytes(X_proj), dev_out >= bytes(dX) + bytes(dW) + bytes(db)
+ * Sizes are rounded up to multiples of 256 bytes per tensor; see rmm_host_staging_bytes().
+ */
+size_t rmm_host_staging_bytes(int64_t N, int64_t D_in, int64_t D_out, int64_t B_proj, rmm_dtype dt,
+                              int backward, int outputs);
+rmm_status rmm_forward_host(const void* X, const void* W, const void* b,
+                            int64_t N, int64_t D_in, int64_t D_out,
+                            uint64_t seed, int64_t B_proj, rmm_dist dist, rmm_dtype dt,
+                            void* Y, void* X_proj,
+                            void* dev_in, void* dev_out,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+rmm_status rmm_backward_host(const void* dY, const void* W, const void* X_proj,
+                             int64_t N, int64_t D_in, int64_t D_out,
+                             uint64_t seed, int64_t B_proj, rmm_dist dist, rmm_dtype dt,
+                             void* dX, void* dW, void* db,
+                             void* dev_in, void* dev_out,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RMM_H_ */

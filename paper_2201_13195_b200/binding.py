@@ -1,0 +1,165 @@
+"""ctypes binding of librmm.so (include/rmm.h): argument marshalling only.
+
+Every step of the layer runs in the CUDA kernels of the library; PyTorch is used here
+for device memory and streams.  There is no fallback: if the library has not been
+built, importing this module raises.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librmm.so")
+
+RMM_OK, RMM_ERR_INVALID_ARG, RMM_ERR_UNSUPPORTED, RMM_ERR_WORKSPACE, RMM_ERR_CUDA, RMM_ERR_TIMEOUT = range(6)
+RMM_DIST_GAUSSIAN, RMM_DIST_RADEMACHER, RMM_DIST_IDENTITY = 0, 1, 2
+RMM_DTYPE_BF16, RMM_DTYPE_F32 = 0, 1
+
+EXPORTS = ("rmm_workspace_bytes", "rmm_forward", "rmm_backward", "rmm_debug_generate_s",
+           "rmm_last_device_status", "rmm_status_string", "rmm_host_staging_bytes",
+           "rmm_forward_host", "rmm_backward_host")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2201_13195_b200.build` "
+                      "(there is no non-CUDA path)")
+_lib = C.CDLL(LIB_PATH)
+
+_i64, _vp, _u64, _int, _sz = C.c_int64, C.c_void_p, C.c_uint64, C.c_int, C.c_size_t
+_lib.rmm_workspace_bytes.argtypes = [_i64, _i64, _i64, _i64, _int]
+_lib.rmm_workspace_bytes.restype = _sz
+_lib.rmm_forward.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _int, _int, _vp, _vp, _vp, _sz, _vp]
+_lib.rmm_forward.restype = _int
+_lib.rmm_backward.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _int, _int, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.rmm_backward.restype = _int
+_lib.rmm_debug_generate_s.argtypes = [_u64, _i64, _i64, _int, _int, _vp, _vp]
+_lib.rmm_debug_generate_s.restype = _int
+_lib.rmm_last_device_status.argtypes = [_vp]
+_lib.rmm_last_device_status.restype = _int
+_lib.rmm_status_string.argtypes = [_int]
+_lib.rmm_status_string.restype = C.c_char_p
+_lib.rmm_host_staging_bytes.argtypes = [_i64, _i64, _i64, _i64, _int, _int, _int]
+_lib.rmm_host_staging_bytes.restype = _sz
+_lib.rmm_forward_host.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _int, _int, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.rmm_forward_host.restype = _int
+_lib.rmm_backward_host.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.rmm_backward_host.restype = _int
+
+
+class RmmError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {rmm_status_string(code)}")
+
+
+def rmm_status_string(code: int) -> str:
+    return _lib.rmm_status_string(int(code)).decode()
+
+
+def _check(code, where):
+    if code != RMM_OK:
+        raise RmmError(code, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return RMM_DTYPE_BF16
+    if t.dtype == torch.float32:
+        return RMM_DTYPE_F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream_ptr(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def rmm_workspace_bytes(N, D_in, D_out, B_proj, dt) -> int:
+    return int(_lib.rmm_workspace_bytes(N, D_in, D_out, B_proj, dt))
+
+
+def alloc_workspace(N, D_in, D_out, B_proj, dt, device="cuda"):
+    return torch.empty(rmm_workspace_bytes(N, D_in, D_out, B_proj, dt), dtype=torch.uint8, device=device)
+
+
+def rmm_forward(X, W, b, seed, B_proj, dist, Y=None, X_proj=None, workspace=None, stream=None, want_y=True):
+    """(Y, X_proj) = (X W^T + 1 b^T, S^T X); device tensors, contiguous."""
+    N, D_in = X.shape
+    D_out = W.shape[0]
+    dt = _dtype_code(X)
+    assert X.is_cuda and X.is_contiguous() and W.is_contiguous() and W.shape[1] == D_in and W.dtype == X.dtype
+    if want_y and Y is None:
+        Y = torch.empty((N, D_out), dtype=X.dtype, device=X.device)
+    if X_proj is None:
+        X_proj = torch.empty((B_proj, D_in), dtype=X.dtype, device=X.device)
+    if workspace is None:
+        workspace = alloc_workspace(N, D_in, D_out, B_proj, dt, X.device)
+    _check(_lib.rmm_forward(_ptr(X), _ptr(W), _ptr(b), N, D_in, D_out, seed, B_proj, dist, dt,
+                            _ptr(Y) if want_y else None, _ptr(X_proj), _ptr(workspace), workspace.numel(),
+                            _stream_ptr(stream)), "rmm_forward")
+    return Y, X_proj
+
+
+def rmm_backward(dY, W, X_proj, seed, dist, dX=None, dW=None, db=None, workspace=None, stream=None,
+                 want_dx=True, want_db=True):
+    """(dX, dW, db) = (dY W, (S^T dY)^T X_proj, sum_rows dY)."""
+    N, D_out = dY.shape
+    D_in = W.shape[1]
+    B_proj = X_proj.shape[0]
+    dt = _dtype_code(dY)
+    assert dY.is_cuda and dY.is_contiguous() and W.is_contiguous() and X_proj.is_contiguous()
+    if want_dx and dX is None:
+        dX = torch.empty((N, D_in), dtype=dY.dtype, device=dY.device)
+    if dW is None:
+        dW = torch.empty((D_out, D_in), dtype=dY.dtype, device=dY.device)
+    if want_db and db is None:
+        db = torch.empty((D_out,), dtype=dY.dtype, device=dY.device)
+    if workspace is None:
+        workspace = alloc_workspace(N, D_in, D_out, B_proj, dt, dY.device)
+    _check(_lib.rmm_backward(_ptr(dY), _ptr(W), _ptr(X_proj), N, D_in, D_out, seed, B_proj, dist, dt,
+                             _ptr(dX) if want_dx else None, _ptr(dW), _ptr(db) if want_db else None,
+                             _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "rmm_backward")
+    return dX, dW, db
+
+
+def rmm_debug_generate_s(seed, N, B_proj, dist, dtype=torch.bfloat16, device="cuda", stream=None):
+    """Unscaled sketch entries P [N, B_proj] as the kernels generate them."""
+    out = torch.empty((N, B_proj), dtype=dtype, device=device)
+    _check(_lib.rmm_debug_generate_s(seed, N, B_proj, dist, _dtype_code(out), _ptr(out), _stream_ptr(stream)),
+           "rmm_debug_generate_s")
+    return out
+
+
+def rmm_last_device_status(workspace) -> int:
+    return int(_lib.rmm_last_device_status(_ptr(workspace)))
+
+
+def rmm_host_staging_bytes(N, D_in, D_out, B_proj, dt, backward, outputs) -> int:
+    return int(_lib.rmm_host_staging_bytes(N, D_in, D_out, B_proj, dt, int(backward), int(outputs)))
+
+
+def rmm_forward_host(X, W, b, seed, B_proj, dist, Y, X_proj, dev_in, dev_out, workspace, stream=None):
+    """Host tensors in and out (pinned recommended); copies are part of the call."""
+    N, D_in = X.shape
+    D_out = W.shape[0]
+    dt = _dtype_code(X)
+    assert not X.is_cuda and not Y.is_cuda and dev_in.is_cuda and dev_out.is_cuda
+    _check(_lib.rmm_forward_host(_ptr(X), _ptr(W), _ptr(b), N, D_in, D_out, seed, B_proj, dist, dt, _ptr(Y),
+                                 _ptr(X_proj), _ptr(dev_in), _ptr(dev_out), _ptr(workspace), workspace.numel(),
+                                 _stream_ptr(stream)), "rmm_forward_host")
+    return Y, X_proj
+
+
+def rmm_backward_host(dY, W, X_proj, seed, dist, dX, dW, db, dev_in, dev_out, workspace, stream=None):
+    N, D_out = dY.shape
+    D_in = W.shape[1]
+    B_proj = X_proj.shape[0]
+    dt = _dtype_code(dY)
+    _check(_lib.rmm_backward_host(_ptr(dY), _ptr(W), _ptr(X_proj), N, D_in, D_out, seed, B_proj, dist, dt,
+                                  _ptr(dX), _ptr(dW), _ptr(db), _ptr(dev_in), _ptr(dev_out), _ptr(workspace),
+                                  workspace.numel(), _stream_ptr(stream)), "rmm_backward_host")
+    return dX, dW, db

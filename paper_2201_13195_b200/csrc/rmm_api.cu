@@ -1,0 +1,358 @@
+// C ABI of the RMM linear layer (see include/rmm.h): argument checks, workspace
+// layout, TMA tensor maps and kernel launches.  All arithmetic runs in the kernels.
+#include "../../include/rmm.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "simt_kernels.cuh"
+#include "sketch_rng.cuh"
+#include "tc_gemm.cuh"
+
+namespace {
+
+using namespace rmm;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+inline size_t elem_bytes(rmm_dtype dt) { return dt == RMM_DTYPE_BF16 ? 2 : 4; }
+
+// ------------------------------------------------------------------ workspace layout
+struct Workspace {
+  size_t status_off, g_off, dbpart_off, total;
+  int db_rows_per_slice, db_slices;
+};
+
+Workspace workspace_layout(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rmm_dtype dt) {
+  (void)D_in;
+  Workspace w;
+  w.status_off = 0;
+  w.g_off = kAlign;
+  size_t off = w.g_off + align_up((size_t)k * (size_t)D_out * elem_bytes(dt));
+  int64_t rps = 256;
+  if ((N + rps - 1) / rps > 256) rps = (N + 255) / 256;
+  w.db_rows_per_slice = (int)rps;
+  w.db_slices = (int)((N + rps - 1) / rps);
+  w.dbpart_off = off;
+  off += align_up((size_t)w.db_slices * (size_t)D_out * sizeof(float));
+  w.total = off;
+  return w;
+}
+
+// ------------------------------------------------------------------ device / driver set-up
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DeviceState {
+  bool ok = false;
+  EncodeTiledFn encode = nullptr;
+};
+
+template <typename K>
+bool allow_big_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+DeviceState& device_state() {
+  static DeviceState st;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    int dev = 0, major = 0, minor = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return;
+    if (cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess) return;
+    if (major != 10) return;  // the kernels are sm_100a only; there is no other path
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || fn == nullptr)
+      return;
+    st.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    bool a = true;
+    a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_K, 4>, tc::GEMM_SMEM_BYTES);
+    a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_MN, 4>, tc::GEMM_SMEM_BYTES);
+    a &= allow_big_smem(tc::gemm_kernel<tc::A_MN, tc::B_MN, 4>, tc::GEMM_SMEM_BYTES);
+    a &= allow_big_smem(tc::gemm_kernel<tc::A_GEN, tc::B_MN, 8>, tc::GEMM_SMEM_BYTES);
+    st.ok = a;
+  });
+  return st;
+}
+
+// Tensor map of a row-major bf16 matrix [rows][cols] (cols contiguous), box = [box_rows][64 cols],
+// 128-byte swizzle, out-of-range elements read as zero.
+bool make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t gstride[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1u, 1u};
+  return device_state().encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box,
+                               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// ------------------------------------------------------------------ launches
+// One contraction on the tensor cores.  a/b are row-major bf16 matrices:
+//   A_K : a is [M][K]   A_MN: a is [K][M]   A_GEN: a unused
+//   B_K : b is [N][K]   B_MN: b is [K][N]
+template <int AMODE, int BMODE>
+rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, int64_t M, int64_t N, int64_t K,
+                     float alpha, int dist, const PhiloxKey& pk, int* status, cudaStream_t stream) {
+  CUtensorMap tmA, tmB;
+  memset(&tmA, 0, sizeof(tmA));
+  bool ok = true;
+  if (AMODE == tc::A_K) ok &= make_tmap(&tmA, a, M, K, tc::BM);
+  if (AMODE == tc::A_MN) ok &= make_tmap(&tmA, a, K, M, tc::BK);
+  if (BMODE == tc::B_K) ok &= make_tmap(&tmB, b, N, K, tc::BN);
+  if (BMODE == tc::B_MN) ok &= make_tmap(&tmB, b, K, N, tc::BK);
+  if (!ok) return RMM_ERR_CUDA;
+  tc::GemmParams p;
+  p.M = M; p.N = N; p.K = K;
+  p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.dist = dist; p.status = status;
+  constexpr int NEPI = (AMODE == tc::A_GEN) ? 8 : 4;
+  dim3 grid((unsigned)((M + tc::BM - 1) / tc::BM), (unsigned)((N + tc::BN - 1) / tc::BN));
+  tc::gemm_kernel<AMODE, BMODE, NEPI><<<grid, 64 + 32 * NEPI, tc::GEMM_SMEM_BYTES, stream>>>(tmA, tmB, p, pk);
+  return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+
+template <typename T, bool GEN_A>
+rmm_status launch_simt(const SimtGemmArgs& g, const PhiloxKey& pk, cudaStream_t stream) {
+  dim3 grid((unsigned)((g.N + SIMT_BN - 1) / SIMT_BN), (unsigned)((g.M + SIMT_BM - 1) / SIMT_BM));
+  simt_gemm_kernel<T, GEN_A><<<grid, SIMT_THREADS, 0, stream>>>(g, pk);
+  return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+
+rmm_status simt_gemm_f32(bool gen_a, const void* A, int64_t a_sm, int64_t a_sk, const void* B, int64_t b_sn,
+                         int64_t b_sk, void* C, const void* bias, int64_t M, int64_t N, int64_t K, float alpha,
+                         int dist, const PhiloxKey& pk, cudaStream_t stream) {
+  SimtGemmArgs g;
+  g.A = A; g.a_sm = a_sm; g.a_sk = a_sk;
+  g.B = B; g.b_sn = b_sn; g.b_sk = b_sk;
+  g.C = C; g.ldc = N; g.bias = bias;
+  g.M = M; g.N = N; g.K = K; g.alpha = alpha; g.dist = dist;
+  return gen_a ? launch_simt<float, true>(g, pk, stream) : launch_simt<float, false>(g, pk, stream);
+}
+
+template <typename T>
+rmm_status launch_db(const void* dY, int64_t N, int64_t D_out, const Workspace& w, char* ws, void* db,
+                     cudaStream_t stream) {
+  float* partial = reinterpret_cast<float*>(ws + w.dbpart_off);
+  dim3 grid((unsigned)((D_out + 255) / 256), (unsigned)w.db_slices);
+  db_partial_kernel<T><<<grid, 256, 0, stream>>>(reinterpret_cast<const T*>(dY), N, D_out, w.db_rows_per_slice, partial);
+  db_finish_kernel<T><<<(unsigned)((D_out + 255) / 256), 256, 0, stream>>>(partial, w.db_slices, D_out,
+                                                                           reinterpret_cast<T*>(db));
+  return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------ argument checks
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+rmm_status check_common(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rmm_dist dist, rmm_dtype dt) {
+  if (N < 1 || D_in < 1 || D_out < 1 || k < 1 || k > N) return RMM_ERR_INVALID_ARG;
+  if (N > (int64_t)1 << 31 || D_in > (int64_t)1 << 30 || D_out > (int64_t)1 << 30) return RMM_ERR_INVALID_ARG;
+  if (dist != RMM_DIST_GAUSSIAN && dist != RMM_DIST_RADEMACHER && dist != RMM_DIST_IDENTITY) return RMM_ERR_INVALID_ARG;
+  if (dt != RMM_DTYPE_BF16 && dt != RMM_DTYPE_F32) return RMM_ERR_INVALID_ARG;
+  if (dist == RMM_DIST_IDENTITY && k != N) return RMM_ERR_INVALID_ARG;
+  if (dt == RMM_DTYPE_BF16 && (D_in % 8 != 0 || D_out % 8 != 0)) return RMM_ERR_UNSUPPORTED;
+  return RMM_OK;
+}
+
+rmm_status check_workspace(const void* ws, size_t ws_bytes, const Workspace& w) {
+  if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0) return RMM_ERR_WORKSPACE;
+  if (ws_bytes < w.total) return RMM_ERR_WORKSPACE;
+  return RMM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t rmm_workspace_bytes(int64_t N, int64_t D_in, int64_t D_out, int64_t B_proj, rmm_dtype dt) {
+  if (N < 1 || D_in < 1 || D_out < 1 || B_proj < 1 || B_proj > N) return 0;
+  if (dt != RMM_DTYPE_BF16 && dt != RMM_DTYPE_F32) return 0;
+  return workspace_layout(N, D_in, D_out, B_proj, dt).total;
+}
+
+rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, int64_t D_in, int64_t D_out,
+                       uint64_t seed, int64_t B_proj, rmm_dist dist, rmm_dtype dt, void* Y, void* X_proj,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  rmm_status st = check_common(N, D_in, D_out, B_proj, dist, dt);
+  if (st != RMM_OK) return st;
+  if (!X || !W || !X_proj) return RMM_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(b) || !aligned16(Y) || !aligned16(X_proj)) return RMM_ERR_INVALID_ARG;
+  const Workspace w = workspace_layout(N, D_in, D_out, B_proj, dt);
+  if ((st = check_workspace(workspace, workspace_bytes, w)) != RMM_OK) return st;
+  if (!device_state().ok) return RMM_ERR_CUDA;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* ws = reinterpret_cast<char*>(workspace);
+  int* status = reinterpret_cast<int*>(ws + w.status_off);
+  if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return RMM_ERR_CUDA;
+  const PhiloxKey pk = make_philox_key(seed);
+  const float c = sketch_scale(B_proj, dist);
+
+  if (dt == RMM_DTYPE_BF16) {
+    if (Y) {
+      st = launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, 0, pk, status, stream);
+      if (st != RMM_OK) return st;
+    }
+    return launch_tc<tc::A_GEN, tc::B_MN>(nullptr, X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, status, stream);
+  }
+  if (Y) {
+    st = simt_gemm_f32(false, X, D_in, 1, W, D_in, 1, Y, b, N, D_out, D_in, 1.0f, 0, pk, stream);
+    if (st != RMM_OK) return st;
+  }
+  return simt_gemm_f32(true, nullptr, 0, 0, X, 1, D_in, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, stream);
+}
+
+rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64_t N, int64_t D_in, int64_t D_out,
+                        uint64_t seed, int64_t B_proj, rmm_dist dist, rmm_dtype dt, void* dX, void* dW, void* db,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  rmm_status st = check_common(N, D_in, D_out, B_proj, dist, dt);
+  if (st != RMM_OK) return st;
+  if (!dY || !W || !X_proj || !dW) return RMM_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(W) || !aligned16(X_proj) || !aligned16(dX) || !aligned16(dW) || !aligned16(db))
+    return RMM_ERR_INVALID_ARG;
+  const Workspace w = workspace_layout(N, D_in, D_out, B_proj, dt);
+  if ((st = check_workspace(workspace, workspace_bytes, w)) != RMM_OK) return st;
+  if (!device_state().ok) return RMM_ERR_CUDA;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* ws = reinterpret_cast<char*>(workspace);
+  int* status = reinterpret_cast<int*>(ws + w.status_off);
+  void* G = ws + w.g_off;
+  if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return RMM_ERR_CUDA;
+  const PhiloxKey pk = make_philox_key(seed);
+  const float c = sketch_scale(B_proj, dist);
+
+  if (dt == RMM_DTYPE_BF16) {
+    if (dX) {
+      st = launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, 0, pk, status, stream);
+      if (st != RMM_OK) return st;
+    }
+    st = launch_tc<tc::A_GEN, tc::B_MN>(nullptr, dY, G, nullptr, B_proj, D_out, N, c, dist, pk, status, stream);
+    if (st != RMM_OK) return st;
+    st = launch_tc<tc::A_MN, tc::B_MN>(G, X_proj, dW, nullptr, D_out, D_in, B_proj, 1.0f, 0, pk, status, stream);
+    if (st != RMM_OK) return st;
+    if (db) return launch_db<__nv_bfloat16>(dY, N, D_out, w, ws, db, stream);
+    return RMM_OK;
+  }
+  if (dX) {
+    st = simt_gemm_f32(false, dY, D_out, 1, W, 1, D_in, dX, nullptr, N, D_in, D_out, 1.0f, 0, pk, stream);
+    if (st != RMM_OK) return st;
+  }
+  st = simt_gemm_f32(true, nullptr, 0, 0, dY, 1, D_out, G, nullptr, B_proj, D_out, N, c, dist, pk, stream);
+  if (st != RMM_OK) return st;
+  st = simt_gemm_f32(false, G, 1, D_out, X_proj, 1, D_in, dW, nullptr, D_out, D_in, B_proj, 1.0f, 0, pk, stream);
+  if (st != RMM_OK) return st;
+  if (db) return launch_db<float>(dY, N, D_out, w, ws, db, stream);
+  return RMM_OK;
+}
+
+rmm_status rmm_debug_generate_s(uint64_t seed, int64_t N, int64_t B_proj, rmm_dist dist, rmm_dtype dt, void* S_out,
+                                void* cuda_stream) {
+  if (N < 1 || B_proj < 1 || B_proj > N || !S_out) return RMM_ERR_INVALID_ARG;
+  if (dist != RMM_DIST_GAUSSIAN && dist != RMM_DIST_RADEMACHER && dist != RMM_DIST_IDENTITY) return RMM_ERR_INVALID_ARG;
+  if (dt != RMM_DTYPE_BF16 && dt != RMM_DTYPE_F32) return RMM_ERR_INVALID_ARG;
+  if (dist == RMM_DIST_IDENTITY && B_proj != N) return RMM_ERR_INVALID_ARG;
+  if (!device_state().ok) return RMM_ERR_CUDA;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const PhiloxKey pk = make_philox_key(seed);
+  const int64_t total = N * B_proj;
+  const unsigned blocks = (unsigned)((total + 255) / 256);
+  if (dt == RMM_DTYPE_BF16)
+    dump_sketch_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(pk, (int)dist, N, B_proj,
+                                                                  reinterpret_cast<__nv_bfloat16*>(S_out));
+  else
+    dump_sketch_kernel<float><<<blocks, 256, 0, stream>>>(pk, (int)dist, N, B_proj, reinterpret_cast<float*>(S_out));
+  return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+
+rmm_status rmm_last_device_status(const void* workspace) {
+  if (!workspace) return RMM_ERR_INVALID_ARG;
+  int v = 0;
+  if (cudaMemcpy(&v, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RMM_ERR_CUDA;
+  return v == 0 ? RMM_OK : RMM_ERR_TIMEOUT;
+}
+
+const char* rmm_status_string(rmm_status s) {
+  switch (s) {
+    case RMM_OK: return "RMM_OK";
+    case RMM_ERR_INVALID_ARG: return "RMM_ERR_INVALID_ARG";
+    case RMM_ERR_UNSUPPORTED: return "RMM_ERR_UNSUPPORTED";
+    case RMM_ERR_WORKSPACE: return "RMM_ERR_WORKSPACE";
+    case RMM_ERR_CUDA: return "RMM_ERR_CUDA";
+    case RMM_ERR_TIMEOUT: return "RMM_ERR_TIMEOUT";
+  }
+  return "RMM_ERR_UNKNOWN";
+}
+
+// ------------------------------------------------------------------ host-buffer wrappers
+size_t rmm_host_staging_bytes(int64_t N, int64_t D_in, int64_t D_out, int64_t B_proj, rmm_dtype dt, int backward,
+                              int outputs) {
+  if (N < 1 || D_in < 1 || D_out < 1 || B_proj < 1) return 0;
+  const size_t e = elem_bytes(dt);
+  const size_t x = align_up((size_t)N * D_in * e), w = align_up((size_t)D_out * D_in * e), bb = align_up((size_t)D_out * e);
+  const size_t y = align_up((size_t)N * D_out * e), xp = align_up((size_t)B_proj * D_in * e);
+  if (!backward) return outputs ? y + xp : x + w + bb;
+  return outputs ? x + w + bb : y + w + xp;
+}
+
+rmm_status rmm_forward_host(const void* X, const void* W, const void* b, int64_t N, int64_t D_in, int64_t D_out,
+                            uint64_t seed, int64_t B_proj, rmm_dist dist, rmm_dtype dt, void* Y, void* X_proj,
+                            void* dev_in, void* dev_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  rmm_status st = check_common(N, D_in, D_out, B_proj, dist, dt);
+  if (st != RMM_OK) return st;
+  if (!X || !W || !X_proj || !dev_in || !dev_out) return RMM_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const size_t e = elem_bytes(dt);
+  const size_t xb = (size_t)N * D_in * e, wb = (size_t)D_out * D_in * e, bb = (size_t)D_out * e;
+  const size_t yb = (size_t)N * D_out * e, xpb = (size_t)B_proj * D_in * e;
+  char* di = reinterpret_cast<char*>(dev_in);
+  char* dout = reinterpret_cast<char*>(dev_out);
+  char *dX = di, *dWt = dX + align_up(xb), *dB = dWt + align_up(wb);
+  char *dYv = dout, *dXp = dYv + align_up(yb);
+  bool ok = cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(dWt, W, wb, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (b) ok = ok && cudaMemcpyAsync(dB, b, bb, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (!ok) return RMM_ERR_CUDA;
+  st = rmm_forward(dX, dWt, b ? dB : nullptr, N, D_in, D_out, seed, B_proj, dist, dt, Y ? dYv : nullptr, dXp,
+                   workspace, workspace_bytes, cuda_stream);
+  if (st != RMM_OK) return st;
+  if (Y) ok = ok && cudaMemcpyAsync(Y, dYv, yb, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(X_proj, dXp, xpb, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  return ok ? RMM_OK : RMM_ERR_CUDA;
+}
+
+rmm_status rmm_backward_host(const void* dY, const void* W, const void* X_proj, int64_t N, int64_t D_in,
+                             int64_t D_out, uint64_t seed, int64_t B_proj, rmm_dist dist, rmm_dtype dt, void* dX,
+                             void* dW, void* db, void* dev_in, void* dev_out, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream) {
+  rmm_status st = check_common(N, D_in, D_out, B_proj, dist, dt);
+  if (st != RMM_OK) return st;
+  if (!dY || !W || !X_proj || !dW || !dev_in || !dev_out) return RMM_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const size_t e = elem_bytes(dt);
+  const size_t xb = (size_t)N * D_in * e, wb = (size_t)D_out * D_in * e, bb = (size_t)D_out * e;
+  const size_t yb = (size_t)N * D_out * e, xpb = (size_t)B_proj * D_in * e;
+  char* di = reinterpret_cast<char*>(dev_in);
+  char* dout = reinterpret_cast<char*>(dev_out);
+  char *ddY = di, *dWt = ddY + align_up(yb), *dXp = dWt + align_up(wb);
+  char *ddX = dout, *ddW = ddX + align_up(xb), *ddb = ddW + align_up(wb);
+  bool ok = cudaMemcpyAsync(ddY, dY, yb, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(dWt, W, wb, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(dXp, X_proj, xpb, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (!ok) return RMM_ERR_CUDA;
+  st = rmm_backward(ddY, dWt, dXp, N, D_in, D_out, seed, B_proj, dist, dt, dX ? ddX : nullptr, ddW, db ? ddb : nullptr,
+                    workspace, workspace_bytes, cuda_stream);
+  if (st != RMM_OK) return st;
+  if (dX) ok = ok && cudaMemcpyAsync(dX, ddX, xb, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(dW, ddW, wb, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  if (db) ok = ok && cudaMemcpyAsync(db, ddb, bb, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  return ok ? RMM_OK : RMM_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,96 @@
+"""Host-side checks that need no GPU: the library loads, exports every symbol that
+include/rmm.h declares, sizes its workspace sensibly and rejects bad arguments with the
+documented codes before anything is launched."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+LIB = os.path.join(ROOT, "paper_2201_13195_b200", "librmm.so")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    if not os.path.exists(LIB):
+        import paper_2201_13195_b200.build as B
+        B.build()
+    return C.CDLL(LIB)
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "rmm.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rmm_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert {"rmm_forward", "rmm_backward", "rmm_workspace_bytes", "rmm_debug_generate_s",
+            "rmm_last_device_status", "rmm_status_string"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_binding_exports_match_header():
+    import paper_2201_13195_b200 as P
+    assert sorted(P.EXPORTS) == _declared_symbols()
+    for n in P.EXPORTS:
+        assert callable(getattr(P, n))
+
+
+def test_status_strings(lib):
+    lib.rmm_status_string.restype = C.c_char_p
+    names = [lib.rmm_status_string(i).decode() for i in range(6)]
+    assert names == ["RMM_OK", "RMM_ERR_INVALID_ARG", "RMM_ERR_UNSUPPORTED", "RMM_ERR_WORKSPACE", "RMM_ERR_CUDA",
+                     "RMM_ERR_TIMEOUT"]
+
+
+def test_workspace_bytes(lib):
+    f = lib.rmm_workspace_bytes
+    f.restype = C.c_size_t
+    f.argtypes = [C.c_int64] * 4 + [C.c_int]
+    big = f(16384, 1024, 4096, 1638, 0)
+    assert big >= 1638 * 4096 * 2 and big % 256 == 0          # holds G = S^T dY in bf16
+    assert f(16384, 1024, 4096, 1638, 1) >= 1638 * 4096 * 4
+    assert f(0, 8, 8, 1, 0) == 0 and f(8, 8, 8, 9, 0) == 0 and f(8, 8, 8, 1, 7) == 0
+
+
+def test_argument_errors_are_reported_before_any_launch(lib):
+    i64, vp = C.c_int64, C.c_void_p
+    fwd = lib.rmm_forward
+    fwd.argtypes = [vp, vp, vp, i64, i64, i64, C.c_uint64, i64, C.c_int, C.c_int, vp, vp, vp, C.c_size_t, vp]
+    bwd = lib.rmm_backward
+    bwd.argtypes = [vp, vp, vp, i64, i64, i64, C.c_uint64, i64, C.c_int, C.c_int, vp, vp, vp, vp, C.c_size_t, vp]
+    p = 4096  # a non-null, 16-byte aligned fake pointer: must never be dereferenced on the host
+    INVALID, UNSUPPORTED, WORKSPACE = 1, 2, 3
+    assert fwd(None, p, None, 8, 8, 8, 0, 4, 0, 0, p, p, p, 1 << 20, None) == INVALID       # null X
+    assert fwd(p, p, None, 8, 8, 8, 0, 9, 0, 0, p, p, p, 1 << 20, None) == INVALID          # B_proj > N
+    assert fwd(p, p, None, 8, 8, 8, 0, 0, 0, 0, p, p, p, 1 << 20, None) == INVALID          # B_proj < 1
+    assert fwd(p, p, None, 8, 8, 8, 0, 4, 5, 0, p, p, p, 1 << 20, None) == INVALID          # bad dist
+    assert fwd(p, p, None, 8, 8, 8, 0, 4, 0, 3, p, p, p, 1 << 20, None) == INVALID          # bad dtype
+    assert fwd(p, p, None, 8, 8, 8, 0, 4, 2, 0, p, p, p, 1 << 20, None) == INVALID          # identity needs k == N
+    assert fwd(p + 4, p, None, 8, 8, 8, 0, 4, 0, 0, p, p, p, 1 << 20, None) == INVALID      # misaligned X
+    assert fwd(p, p, None, 8, 12, 8, 0, 4, 0, 0, p, p, p, 1 << 20, None) == UNSUPPORTED     # D_in % 8 in bf16
+    assert fwd(p, p, None, 8, 8, 8, 0, 4, 0, 0, p, p, None, 0, None) == WORKSPACE           # no workspace
+    assert fwd(p, p, None, 8, 8, 8, 0, 4, 0, 0, p, p, p, 16, None) == WORKSPACE             # too small
+    assert fwd(p, p, None, 8, 8, 8, 0, 4, 0, 0, p, p, p + 16, 1 << 20, None) == WORKSPACE   # misaligned workspace
+    assert bwd(p, p, p, 8, 8, 8, 0, 4, 0, 0, p, None, p, p, 1 << 20, None) == INVALID       # dW is required
+    assert bwd(p, p, p, 8, 8, 8, 0, 4, 0, 0, p, p, p, None, 0, None) == WORKSPACE
+    gen = lib.rmm_debug_generate_s
+    gen.argtypes = [C.c_uint64, i64, i64, C.c_int, C.c_int, vp, vp]
+    assert gen(0, 8, 9, 0, 0, p, None) == INVALID
+    assert gen(0, 8, 4, 0, 0, None, None) == INVALID
+
+
+def test_no_device_is_an_error_not_a_fallback(lib):
+    """Without a usable sm_100a device a well-formed call must fail with RMM_ERR_CUDA."""
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present")
+    i64, vp = C.c_int64, C.c_void_p
+    fwd = lib.rmm_forward
+    fwd.argtypes = [vp, vp, vp, i64, i64, i64, C.c_uint64, i64, C.c_int, C.c_int, vp, vp, vp, C.c_size_t, vp]
+    p = 4096
+    assert fwd(p, p, None, 8, 8, 8, 0, 4, 0, 0, p, p, p, 1 << 20, None) == 4
