@@ -1,0 +1,334 @@
+#!/usr/bin/env python
+"""Benchmark of the RMM linear layer (forward + backward through the C ABI) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = rmm_forward + rmm_backward on one batch of synthetic, seeded input of the
+named workload.  Prints ONE JSON line.  With N > 1 (launched under torchrun) every rank
+runs an independent replica of the same layer (the path does not shard); the value is
+the aggregate over ranks, timed on the device, maximum over ranks.
+
+--impl reference times the CPU fp64 oracle (oracle/) on this machine's host cores, on a
+bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import rmm_inputs as R  # noqa: E402
+
+METRIC = "RMM linear fwd+bwd TFLOP/s (bf16)"
+UNIT = "TFLOP/s"
+DEFAULT_WORKLOAD = "large_ffn_up_rho0.1"
+STEP_ORDER = ("y", "sketch", "dx", "sdy", "dw", "db")
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index, period=0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons = [], set()
+        self.stop_flag = threading.Event()
+        self.max_mhz = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap,
+                 "hw_power_brake": nv.nvmlClocksThrottleReasonHwPowerBrakeSlowdown}
+        while not self.stop_flag.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def result(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+# ----------------------------------------------------------------------------- oracle legs
+def oracle_sample_seconds(w, n_tokens):
+    """One forward+backward of the oracle on the first n_tokens rows (same rho); returns (seconds, flops)."""
+    from oracle import oracle as O
+    ws = R.Workload(w.name, w.dtype, n_tokens, w.d_in, w.d_out, w.rho, w.dist, w.seed, w.x_std, w.w_std, w.dy_std)
+    X, W, b, dY = R.make_inputs(w, n_tokens=n_tokens)
+    X, W, dY = X.astype(np.float64), W.astype(np.float64), dY.astype(np.float64)
+    store = O.STORE_BF16 if w.dtype == R.DTYPE_BF16 else O.STORE_F32
+    t0 = time.perf_counter()
+    S = O.generate_s(ws.seed, n_tokens, ws.b_proj, ws.dist, store)
+    _, Xp = O.forward(X, W, None, S)
+    O.backward(dY, W, Xp, S)
+    dt = time.perf_counter() - t0
+    return dt, ws.flops()["total"], ws.b_proj
+
+
+def pick_sample_tokens(w, budget_s):
+    """Token count whose oracle pass should take about budget_s, from a small calibration pass."""
+    n0 = min(w.n_tokens, 128)
+    t, f, _ = oracle_sample_seconds(w, n0)
+    rate = f / max(t, 1e-6)
+    n = n0
+    while n * 2 <= w.n_tokens:
+        ws = R.Workload(w.name, w.dtype, n * 2, w.d_in, w.d_out, w.rho, w.dist, w.seed)
+        if ws.flops()["total"] / rate > budget_s:
+            break
+        n *= 2
+    return n
+
+
+def cpu_baseline(w, budget_s=15.0):
+    from oracle import oracle as O
+    n = pick_sample_tokens(w, budget_s)
+    t, f, k = oracle_sample_seconds(w, n)
+    return {"value": f / t / 1e12, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"first {n} of {w.n_tokens} token rows, B_proj = {k} (same rho), one fwd+bwd in {t:.2f} s",
+            "seconds": t}
+
+
+def run_reference(args, w):
+    """The reference arm: the oracle as it stands on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle as O
+    total_budget = 120.0
+    per_step = total_budget / max(1, args.steps + args.warmup)
+    n = pick_sample_tokens(w, per_step)
+    for _ in range(args.warmup):
+        oracle_sample_seconds(w, n)
+    ts, fl, k = [], 0, 0
+    for _ in range(args.steps):
+        t, fl, k = oracle_sample_seconds(w, n)
+        ts.append(t)
+    tot = float(np.sum(ts))
+    value = fl * args.steps / tot / 1e12
+    sample = f"first {n} of {w.n_tokens} token rows, B_proj = {k} (same rho) per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w):
+    touched = (2 * w.n_tokens * (w.d_in + w.d_out) * 2 + 3 * w.d_in * w.d_out + 2 * w.b_proj * (w.d_in + w.d_out)) * w.elem_bytes
+    return {"workload": w.name, "n_tokens": w.n_tokens, "d_in": w.d_in, "d_out": w.d_out, "rho": w.rho,
+            "b_proj": w.b_proj, "sketch": ("gaussian", "rademacher", "identity")[w.dist], "seed": w.seed,
+            "l2": f"inputs larger than L2: about {touched / 1e6:.0f} MB of tensors touched per step, no flush"}
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(R.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = R.WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2201_13195_b200 as P
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    # ---- inputs, resident in HBM before the timed region
+    X, W, b, dY = R.make_inputs(w)
+    td = torch.bfloat16 if w.dtype == R.DTYPE_BF16 else torch.float32
+    Xd, Wd, dYd = [torch.from_numpy(a).cuda().to(td).contiguous() for a in (X, W, dY)]
+    N, k = w.n_tokens, w.b_proj
+    Y = torch.empty((N, w.d_out), dtype=td, device="cuda")
+    Xp = torch.empty((k, w.d_in), dtype=td, device="cuda")
+    dX = torch.empty((N, w.d_in), dtype=td, device="cuda")
+    dW = torch.empty((w.d_out, w.d_in), dtype=td, device="cuda")
+    db = torch.empty((w.d_out,), dtype=td, device="cuda")
+    ws = P.alloc_workspace(N, w.d_in, w.d_out, k, w.dtype)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        seed = w.seed + i          # a fresh S every step (Algorithm 1)
+        P.rmm_forward(Xd, Wd, None, seed, k, w.dist, Y=Y, X_proj=Xp, workspace=ws, stream=stream)
+        P.rmm_backward(dYd, Wd, Xp, seed, w.dist, dX=dX, dW=dW, db=db, workspace=ws, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    assert P.rmm_last_device_status(ws) == P.RMM_OK
+
+    launches_per_step = 7
+    P.rmm_profile_enable(min(args.steps, 200) * 6)     # per-kernel events for the first 200 timed steps
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i)
+    e1.record(stream)
+    barrier()
+    sampler.stop_flag.set()
+    sampler.join()
+    ms_total = e0.elapsed_time(e1)
+    assert P.rmm_last_device_status(ws) == P.RMM_OK
+    records = P.rmm_profile_read(min(args.steps, 200) * 6)
+    P.rmm_profile_enable(0)
+
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    fl = w.flops()
+    value = world * fl["total"] / (ms_step * 1e-3) / 1e12
+
+    # ---- per-kernel durations and roofline of the dominant kernel
+    per_kernel = {}
+    for name in STEP_ORDER:
+        v = [ms for n, ms in records if n == name]
+        if v:
+            per_kernel[name] = {"ms": float(np.mean(v)), "launches_timed": len(v)}
+    peaks = load_peaks()
+    flops_of = {"y": fl["y"], "sketch": fl["sketch"], "dx": fl["dx"], "sdy": fl["sdy"], "dw": fl["dw"]}
+    for name, d in per_kernel.items():
+        if name in flops_of:
+            d["tflops"] = flops_of[name] / (d["ms"] * 1e-3) / 1e12
+    dom = max((n for n in per_kernel if n in flops_of), key=lambda n: per_kernel[n]["ms"])
+    achieved = per_kernel[dom]["tflops"]
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
+                "peak_kind": f"sustained bf16 GEMM, of {peaks['source']}", "frac_of_burst": achieved / peaks["bf16_tflops"],
+                "traffic": None, "algorithmic_flops_per_launch": flops_of[dom]}
+
+    # ---- end to end through the host-buffer entry points (pinned host memory)
+    e2e = None
+    if rank == 0 or world > 1:
+        hX, hW, hdY = [torch.from_numpy(a).to(td).pin_memory() for a in (X, W, dY)]
+        hY, hXp = torch.empty_like(Y, device="cpu").pin_memory(), torch.empty_like(Xp, device="cpu").pin_memory()
+        hdX, hdW, hdb = [torch.empty_like(a, device="cpu").pin_memory() for a in (dX, dW, db)]
+        nb = max(P.rmm_host_staging_bytes(N, w.d_in, w.d_out, k, w.dtype, bw, o) for bw in (0, 1) for o in (0, 1))
+        dev_in = torch.empty(nb, dtype=torch.uint8, device="cuda")
+        dev_out = torch.empty(nb, dtype=torch.uint8, device="cuda")
+
+        def e2e_step(i):
+            seed = w.seed + 100000 + i
+            P.rmm_forward_host(hX, hW, None, seed, k, w.dist, hY, hXp, dev_in, dev_out, ws, stream=stream)
+            P.rmm_backward_host(hdY, hW, hXp, seed, w.dist, hdX, hdW, hdb, dev_in, dev_out, ws, stream=stream)
+
+        for i in range(2):
+            e2e_step(i)
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for i in range(args.e2e_steps):
+            e2e_step(2 + i)
+        g1.record(stream)
+        torch.cuda.synchronize()
+        dt = g0.elapsed_time(g1) * 1e-3
+        tt = torch.tensor([dt], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        dt = float(tt.item())
+        eb = w.elem_bytes
+        h2d = (N * w.d_in + w.d_out * w.d_in) * eb + (N * w.d_out + w.d_out * w.d_in + k * w.d_in) * eb
+        d2h = (N * w.d_out + k * w.d_in) * eb + (N * w.d_in + w.d_out * w.d_in + w.d_out) * eb
+        e2e = {"value": world * fl["total"] * args.e2e_steps / dt / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "ms_per_step": 1e3 * dt / args.e2e_steps}
+
+    if rank == 0:
+        cpu = None if args.no_cpu_baseline or world > 1 else cpu_baseline(w)
+        saved = w.saved_bytes()
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16" if w.dtype == R.DTYPE_BF16 else "f32", "data": "synthetic",
+                "config": workload_config(w), "clocks": sampler.result(), "e2e": e2e,
+                "gpu_launches": launches_per_step * args.steps, "roofline": roofline, "cpu_baseline": cpu,
+                "pct_of_tensor_peak": {"burst": 100 * value / world / peaks["bf16_tflops"],
+                                       "sustained": 100 * value / world / peaks["bf16_tflops_sustained"],
+                                       "of": peaks["source"]},
+                "effective_tflops_exact_layer_flops": world * fl["exact_layer"] / (ms_step * 1e-3) / 1e12,
+                "saved_activation_bytes": saved, "workspace_bytes": int(ws.numel()), "per_kernel": per_kernel,
+                "replicas": "independent layers, no collective" if world > 1 else None}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -124,6 +124,28 @@ rmm_status rmm_last_device_status(const void* workspace);
 const char* rmm_status_string(rmm_status s);
 
 /*
+ * Per-kernel timing for benchmarks (no counterpart in the paper).  While enabled,
+ * every kernel that rmm_forward / rmm_backward launch is bracketed by a pair of CUDA
+ * events recorded on the caller's stream, up to `capacity` launches; further launches
+ * are not recorded.  Event objects are created by rmm_profile_enable(capacity > 0)
+ * and destroyed by rmm_profile_enable(0).  Process-wide, not thread-safe; meant for a
+ * single benchmarking thread.
+ *   rmm_profile_read: waits for the recorded events, writes for each recorded launch
+ *   its step id (rmm_step below) and its duration in milliseconds, returns the
+ *   number of records written (at most max_records) and clears the record list.
+ */
+typedef enum {
+  RMM_STEP_Y = 0,       /* Y = X W^T + b            (Eq. 1) */
+  RMM_STEP_SKETCH = 1,  /* X_proj = S^T X           (Section 2.1) */
+  RMM_STEP_DX = 2,      /* dX = dY W                (Eq. 2) */
+  RMM_STEP_SDY = 3,     /* G = S^T dY               (Algorithm 1, inner product of Eq. 4) */
+  RMM_STEP_DW = 4,      /* dW = G^T X_proj          (Eq. 4) */
+  RMM_STEP_DB = 5       /* db = dY^T 1              (Eq. 3), partial sums and final sum */
+} rmm_step;
+rmm_status rmm_profile_enable(int capacity);
+int rmm_profile_read(int* step_ids, float* milliseconds, int max_records);
+
+/*
  * Host-buffer convenience wrappers (end-to-end path): the tensor arguments are HOST
  * pointers (pinned memory recommended); the device buffers dev_* and the workspace
  * are caller-owned DEVICE scratch of at least the tensors' sizes.  Each call copies

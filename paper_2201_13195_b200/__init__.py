@@ -1,6 +1,16 @@
 """B200 (sm_100a) implementation of the randomized-matrix-multiplication linear layer
-of arXiv 2201.13195: a C-ABI CUDA library (include/rmm.h) and its ctypes binding."""
-from .binding import *  # noqa: F401,F403
-from .binding import (EXPORTS, LIB_PATH, RmmError, alloc_workspace, rmm_backward, rmm_backward_host,
-                      rmm_debug_generate_s, rmm_forward, rmm_forward_host, rmm_host_staging_bytes,
-                      rmm_last_device_status, rmm_status_string, rmm_workspace_bytes)
+of arXiv 2201.13195: a C-ABI CUDA library (include/rmm.h) and its ctypes binding.
+
+The binding (and with it librmm.so) is loaded on first use of any attribute, so that
+``python -m paper_2201_13195_b200.build`` can run before the library exists.  There is
+no non-CUDA path: using the package without a built library raises ImportError.
+"""
+import importlib
+
+
+def __getattr__(name):
+    binding = importlib.import_module(".binding", __name__)
+    try:
+        return getattr(binding, name)
+    except AttributeError:
+        raise AttributeError(f"module {__name__!r} has no attribute {name!r}") from None

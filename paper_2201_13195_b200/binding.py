@@ -18,7 +18,8 @@ RMM_DTYPE_BF16, RMM_DTYPE_F32 = 0, 1
 
 EXPORTS = ("rmm_workspace_bytes", "rmm_forward", "rmm_backward", "rmm_debug_generate_s",
            "rmm_last_device_status", "rmm_status_string", "rmm_host_staging_bytes",
-           "rmm_forward_host", "rmm_backward_host")
+           "rmm_forward_host", "rmm_backward_host", "rmm_profile_enable", "rmm_profile_read")
+STEP_NAMES = ("y", "sketch", "dx", "sdy", "dw", "db")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2201_13195_b200.build` "
@@ -44,6 +45,10 @@ _lib.rmm_forward_host.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _
 _lib.rmm_forward_host.restype = _int
 _lib.rmm_backward_host.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.rmm_backward_host.restype = _int
+_lib.rmm_profile_enable.argtypes = [_int]
+_lib.rmm_profile_enable.restype = _int
+_lib.rmm_profile_read.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_float), _int]
+_lib.rmm_profile_read.restype = _int
 
 
 class RmmError(RuntimeError):
@@ -163,3 +168,16 @@ def rmm_backward_host(dY, W, X_proj, seed, dist, dX, dW, db, dev_in, dev_out, wo
                                   _ptr(dX), _ptr(dW), _ptr(db), _ptr(dev_in), _ptr(dev_out), _ptr(workspace),
                                   workspace.numel(), _stream_ptr(stream)), "rmm_backward_host")
     return dX, dW, db
+
+
+def rmm_profile_enable(capacity: int) -> None:
+    """Bracket each kernel launch of the next calls with CUDA events (capacity launches); 0 switches it off."""
+    _check(_lib.rmm_profile_enable(int(capacity)), "rmm_profile_enable")
+
+
+def rmm_profile_read(max_records: int):
+    """[(step name, milliseconds)] of the launches recorded since the last read."""
+    ids = (C.c_int * max_records)()
+    ms = (C.c_float * max_records)()
+    n = _lib.rmm_profile_read(ids, ms, max_records)
+    return [(STEP_NAMES[ids[i]], float(ms[i])) for i in range(n)]

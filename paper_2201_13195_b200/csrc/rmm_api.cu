@@ -7,6 +7,7 @@
 #include <cuda_runtime.h>
 
 #include <mutex>
+#include <vector>
 
 #include "simt_kernels.cuh"
 #include "sketch_rng.cuh"
@@ -93,6 +94,33 @@ bool make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, i
                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+
+// ------------------------------------------------------------------ per-kernel timing (benchmarks)
+struct ProfileRecord { int step; cudaEvent_t t0, t1; };
+struct Profiler {
+  std::vector<ProfileRecord> pool;
+  size_t used = 0;
+};
+Profiler& profiler() {
+  static Profiler p;
+  return p;
+}
+// Brackets the launches made while it is alive with two events on the stream.
+struct ScopedTiming {
+  ProfileRecord* rec = nullptr;
+  cudaStream_t stream;
+  ScopedTiming(int step, cudaStream_t s) : stream(s) {
+    Profiler& p = profiler();
+    if (p.used < p.pool.size()) {
+      rec = &p.pool[p.used++];
+      rec->step = step;
+      cudaEventRecord(rec->t0, stream);
+    }
+  }
+  ~ScopedTiming() {
+    if (rec) cudaEventRecord(rec->t1, stream);
+  }
+};
 
 // ------------------------------------------------------------------ launches
 // One contraction on the tensor cores.  a/b are row-major bf16 matrices:
@@ -195,15 +223,19 @@ rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, i
 
   if (dt == RMM_DTYPE_BF16) {
     if (Y) {
+      ScopedTiming t(RMM_STEP_Y, stream);
       st = launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, 0, pk, status, stream);
       if (st != RMM_OK) return st;
     }
+    ScopedTiming t(RMM_STEP_SKETCH, stream);
     return launch_tc<tc::A_GEN, tc::B_MN>(nullptr, X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, status, stream);
   }
   if (Y) {
+    ScopedTiming t(RMM_STEP_Y, stream);
     st = simt_gemm_f32(false, X, D_in, 1, W, D_in, 1, Y, b, N, D_out, D_in, 1.0f, 0, pk, stream);
     if (st != RMM_OK) return st;
   }
+  ScopedTiming t(RMM_STEP_SKETCH, stream);
   return simt_gemm_f32(true, nullptr, 0, 0, X, 1, D_in, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, stream);
 }
 
@@ -228,25 +260,45 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
 
   if (dt == RMM_DTYPE_BF16) {
     if (dX) {
+      ScopedTiming t(RMM_STEP_DX, stream);
       st = launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, 0, pk, status, stream);
       if (st != RMM_OK) return st;
     }
-    st = launch_tc<tc::A_GEN, tc::B_MN>(nullptr, dY, G, nullptr, B_proj, D_out, N, c, dist, pk, status, stream);
-    if (st != RMM_OK) return st;
-    st = launch_tc<tc::A_MN, tc::B_MN>(G, X_proj, dW, nullptr, D_out, D_in, B_proj, 1.0f, 0, pk, status, stream);
-    if (st != RMM_OK) return st;
-    if (db) return launch_db<__nv_bfloat16>(dY, N, D_out, w, ws, db, stream);
+    {
+      ScopedTiming t(RMM_STEP_SDY, stream);
+      st = launch_tc<tc::A_GEN, tc::B_MN>(nullptr, dY, G, nullptr, B_proj, D_out, N, c, dist, pk, status, stream);
+      if (st != RMM_OK) return st;
+    }
+    {
+      ScopedTiming t(RMM_STEP_DW, stream);
+      st = launch_tc<tc::A_MN, tc::B_MN>(G, X_proj, dW, nullptr, D_out, D_in, B_proj, 1.0f, 0, pk, status, stream);
+      if (st != RMM_OK) return st;
+    }
+    if (db) {
+      ScopedTiming t(RMM_STEP_DB, stream);
+      return launch_db<__nv_bfloat16>(dY, N, D_out, w, ws, db, stream);
+    }
     return RMM_OK;
   }
   if (dX) {
+    ScopedTiming t(RMM_STEP_DX, stream);
     st = simt_gemm_f32(false, dY, D_out, 1, W, 1, D_in, dX, nullptr, N, D_in, D_out, 1.0f, 0, pk, stream);
     if (st != RMM_OK) return st;
   }
-  st = simt_gemm_f32(true, nullptr, 0, 0, dY, 1, D_out, G, nullptr, B_proj, D_out, N, c, dist, pk, stream);
-  if (st != RMM_OK) return st;
-  st = simt_gemm_f32(false, G, 1, D_out, X_proj, 1, D_in, dW, nullptr, D_out, D_in, B_proj, 1.0f, 0, pk, stream);
-  if (st != RMM_OK) return st;
-  if (db) return launch_db<float>(dY, N, D_out, w, ws, db, stream);
+  {
+    ScopedTiming t(RMM_STEP_SDY, stream);
+    st = simt_gemm_f32(true, nullptr, 0, 0, dY, 1, D_out, G, nullptr, B_proj, D_out, N, c, dist, pk, stream);
+    if (st != RMM_OK) return st;
+  }
+  {
+    ScopedTiming t(RMM_STEP_DW, stream);
+    st = simt_gemm_f32(false, G, 1, D_out, X_proj, 1, D_in, dW, nullptr, D_out, D_in, B_proj, 1.0f, 0, pk, stream);
+    if (st != RMM_OK) return st;
+  }
+  if (db) {
+    ScopedTiming t(RMM_STEP_DB, stream);
+    return launch_db<float>(dY, N, D_out, w, ws, db, stream);
+  }
   return RMM_OK;
 }
 
@@ -286,6 +338,42 @@ const char* rmm_status_string(rmm_status s) {
     case RMM_ERR_TIMEOUT: return "RMM_ERR_TIMEOUT";
   }
   return "RMM_ERR_UNKNOWN";
+}
+
+rmm_status rmm_profile_enable(int capacity) {
+  Profiler& p = profiler();
+  for (ProfileRecord& r : p.pool) {
+    cudaEventDestroy(r.t0);
+    cudaEventDestroy(r.t1);
+  }
+  p.pool.clear();
+  p.used = 0;
+  if (capacity <= 0) return RMM_OK;
+  if (!device_state().ok) return RMM_ERR_CUDA;
+  p.pool.reserve((size_t)capacity);
+  for (int i = 0; i < capacity; ++i) {
+    ProfileRecord r;
+    r.step = -1;
+    if (cudaEventCreate(&r.t0) != cudaSuccess) return RMM_ERR_CUDA;
+    if (cudaEventCreate(&r.t1) != cudaSuccess) { cudaEventDestroy(r.t0); return RMM_ERR_CUDA; }
+    p.pool.push_back(r);
+  }
+  return RMM_OK;
+}
+
+int rmm_profile_read(int* step_ids, float* milliseconds, int max_records) {
+  Profiler& p = profiler();
+  int n = 0;
+  for (size_t i = 0; i < p.used && n < max_records; ++i) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(p.pool[i].t1) != cudaSuccess) break;
+    if (cudaEventElapsedTime(&ms, p.pool[i].t0, p.pool[i].t1) != cudaSuccess) break;
+    if (step_ids) step_ids[n] = p.pool[i].step;
+    if (milliseconds) milliseconds[n] = ms;
+    ++n;
+  }
+  p.used = 0;
+  return n;
 }
 
 // ------------------------------------------------------------------ host-buffer wrappers
