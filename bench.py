@@ -115,10 +115,11 @@ def oracle_sample_seconds(w, n_tokens):
 
 
 def pick_sample_tokens(w, budget_s):
-    """Token count whose oracle pass should take about budget_s, from a small calibration pass."""
-    n0 = min(w.n_tokens, 128)
+    """Token count whose oracle pass should take about budget_s, from a small calibration pass.
+    The oracle's strided loops slow down as the sample grows, hence the factor 3 of caution."""
+    n0 = min(w.n_tokens, 256)
     t, f, _ = oracle_sample_seconds(w, n0)
-    rate = f / max(t, 1e-6)
+    rate = f / max(t, 1e-6) / 3.0
     n = n0
     while n * 2 <= w.n_tokens:
         ws = R.Workload(w.name, w.dtype, n * 2, w.d_in, w.d_out, w.rho, w.dist, w.seed)
@@ -128,7 +129,7 @@ def pick_sample_tokens(w, budget_s):
     return n
 
 
-def cpu_baseline(w, budget_s=15.0):
+def cpu_baseline(w, budget_s=20.0):
     from oracle import oracle as O
     n = pick_sample_tokens(w, budget_s)
     t, f, k = oracle_sample_seconds(w, n)
@@ -143,7 +144,7 @@ def run_reference(args, w):
     if rank != 0:
         return
     from oracle import oracle as O
-    total_budget = 120.0
+    total_budget = 90.0
     per_step = total_budget / max(1, args.steps + args.warmup)
     n = pick_sample_tokens(w, per_step)
     for _ in range(args.warmup):

@@ -12,6 +12,7 @@
 #include "simt_kernels.cuh"
 #include "sketch_rng.cuh"
 #include "tc_gemm.cuh"
+#include "tc_sketch.cuh"
 
 namespace {
 
@@ -22,13 +23,14 @@ inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 inline size_t elem_bytes(rmm_dtype dt) { return dt == RMM_DTYPE_BF16 ? 2 : 4; }
 
 // ------------------------------------------------------------------ workspace layout
+// [status word | G = S^T dY | scratch], scratch = fp32 partial tiles of the sketch kernels
+// (bf16 mode) or partial column sums of db (fp32 mode).
 struct Workspace {
-  size_t status_off, g_off, dbpart_off, total;
+  size_t status_off, g_off, scratch_off, total;
   int db_rows_per_slice, db_slices;
 };
 
 Workspace workspace_layout(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rmm_dtype dt) {
-  (void)D_in;
   Workspace w;
   w.status_off = 0;
   w.g_off = kAlign;
@@ -37,8 +39,15 @@ Workspace workspace_layout(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rm
   if ((N + rps - 1) / rps > 256) rps = (N + 255) / 256;
   w.db_rows_per_slice = (int)rps;
   w.db_slices = (int)((N + rps - 1) / rps);
-  w.dbpart_off = off;
-  off += align_up((size_t)w.db_slices * (size_t)D_out * sizeof(float));
+  w.scratch_off = off;
+  size_t scratch = (size_t)w.db_slices * (size_t)D_out * sizeof(float);
+  if (dt == RMM_DTYPE_BF16) {
+    const tc::SketchSchedule f = tc::make_sketch_schedule(k, D_in, N, tc::SK_MAX_CTAS);
+    const tc::SketchSchedule b = tc::make_sketch_schedule(k + 1, D_out, N, tc::SK_MAX_CTAS);
+    const long long slots = f.num_slots() > b.num_slots() ? f.num_slots() : b.num_slots();
+    scratch = (size_t)slots * tc::SK_TILE_ELEMS * sizeof(float);
+  }
+  off += align_up(scratch);
   w.total = off;
   return w;
 }
@@ -51,6 +60,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct DeviceState {
   bool ok = false;
   EncodeTiledFn encode = nullptr;
+  int num_sms = 0;
 };
 
 template <typename K>
@@ -67,6 +77,7 @@ DeviceState& device_state() {
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return;
     if (cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess) return;
     if (major != 10) return;  // the kernels are sm_100a only; there is no other path
+    if (cudaDeviceGetAttribute(&st.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -74,10 +85,10 @@ DeviceState& device_state() {
       return;
     st.encode = reinterpret_cast<EncodeTiledFn>(fn);
     bool a = true;
-    a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_K, 4>, tc::GEMM_SMEM_BYTES);
-    a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_MN, 4>, tc::GEMM_SMEM_BYTES);
-    a &= allow_big_smem(tc::gemm_kernel<tc::A_MN, tc::B_MN, 4>, tc::GEMM_SMEM_BYTES);
-    a &= allow_big_smem(tc::gemm_kernel<tc::A_GEN, tc::B_MN, 8>, tc::GEMM_SMEM_BYTES);
+    a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_K>, tc::GEMM_SMEM_BYTES);
+    a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_MN>, tc::GEMM_SMEM_BYTES);
+    a &= allow_big_smem(tc::gemm_kernel<tc::A_MN, tc::B_MN>, tc::GEMM_SMEM_BYTES);
+    a &= allow_big_smem(tc::sketch_kernel, tc::SK_SMEM_BYTES);
     st.ok = a;
   });
   return st;
@@ -124,13 +135,12 @@ struct ScopedTiming {
 
 // ------------------------------------------------------------------ launches
 // One contraction on the tensor cores.  a/b are row-major bf16 matrices:
-//   A_K : a is [M][K]   A_MN: a is [K][M]   A_GEN: a unused
+//   A_K : a is [M][K]   A_MN: a is [K][M]
 //   B_K : b is [N][K]   B_MN: b is [K][N]
 template <int AMODE, int BMODE>
 rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, int64_t M, int64_t N, int64_t K,
-                     float alpha, int dist, const PhiloxKey& pk, int* status, cudaStream_t stream) {
+                     float alpha, int* status, cudaStream_t stream) {
   CUtensorMap tmA, tmB;
-  memset(&tmA, 0, sizeof(tmA));
   bool ok = true;
   if (AMODE == tc::A_K) ok &= make_tmap(&tmA, a, M, K, tc::BM);
   if (AMODE == tc::A_MN) ok &= make_tmap(&tmA, a, K, M, tc::BK);
@@ -139,10 +149,33 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   if (!ok) return RMM_ERR_CUDA;
   tc::GemmParams p;
   p.M = M; p.N = N; p.K = K;
-  p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.dist = dist; p.status = status;
-  constexpr int NEPI = (AMODE == tc::A_GEN) ? 8 : 4;
+  p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.status = status;
   dim3 grid((unsigned)((M + tc::BM - 1) / tc::BM), (unsigned)((N + tc::BN - 1) / tc::BN));
-  tc::gemm_kernel<AMODE, BMODE, NEPI><<<grid, 64 + 32 * NEPI, tc::GEMM_SMEM_BYTES, stream>>>(tmA, tmB, p, pk);
+  tc::gemm_kernel<AMODE, BMODE><<<grid, 64 + 32 * tc::NEPI, tc::GEMM_SMEM_BYTES, stream>>>(tmA, tmB, p);
+  return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+
+// Sketch contraction out[j][d] = c * sum_n P[n][j] * b[n][d] for j < k (b is [tokens][cols] bf16),
+// and, when ones_out is given, ones_out[d] = sum_n b[n][d] from the extra row of ones.
+rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, int64_t cols, int64_t tokens, float c,
+                         int dist, const PhiloxKey& pk, float* partial, int* status, cudaStream_t stream) {
+  CUtensorMap tmB;
+  if (!make_tmap(&tmB, b, tokens, cols, tc::SK_BK)) return RMM_ERR_CUDA;
+  tc::SketchParams p;
+  p.rows = k + (ones_out ? 1 : 0);
+  p.b_proj = k;
+  p.cols = cols;
+  p.tokens = tokens;
+  p.partial = partial;
+  p.dist = dist;
+  p.ones_row = ones_out ? 1 : 0;
+  p.status = status;
+  const int sms = device_state().num_sms;
+  p.sched = tc::make_sketch_schedule(p.rows, cols, tokens, sms < tc::SK_MAX_CTAS ? sms : tc::SK_MAX_CTAS);
+  tc::sketch_kernel<<<p.sched.num_ctas, tc::SK_THREADS, tc::SK_SMEM_BYTES, stream>>>(tmB, p, pk);
+  dim3 rgrid((unsigned)(p.sched.tiles_m * p.sched.tiles_n), tc::SK_BM / tc::SKR_ROWS);
+  tc::sketch_reduce_kernel<<<rgrid, 128, 0, stream>>>(p, c, reinterpret_cast<__nv_bfloat16*>(out),
+                                                      reinterpret_cast<__nv_bfloat16*>(ones_out));
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
 
@@ -167,7 +200,7 @@ rmm_status simt_gemm_f32(bool gen_a, const void* A, int64_t a_sm, int64_t a_sk, 
 template <typename T>
 rmm_status launch_db(const void* dY, int64_t N, int64_t D_out, const Workspace& w, char* ws, void* db,
                      cudaStream_t stream) {
-  float* partial = reinterpret_cast<float*>(ws + w.dbpart_off);
+  float* partial = reinterpret_cast<float*>(ws + w.scratch_off);
   dim3 grid((unsigned)((D_out + 255) / 256), (unsigned)w.db_slices);
   db_partial_kernel<T><<<grid, 256, 0, stream>>>(reinterpret_cast<const T*>(dY), N, D_out, w.db_rows_per_slice, partial);
   db_finish_kernel<T><<<(unsigned)((D_out + 255) / 256), 256, 0, stream>>>(partial, w.db_slices, D_out,
@@ -224,11 +257,12 @@ rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, i
   if (dt == RMM_DTYPE_BF16) {
     if (Y) {
       ScopedTiming t(RMM_STEP_Y, stream);
-      st = launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, 0, pk, status, stream);
+      st = launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, status, stream);
       if (st != RMM_OK) return st;
     }
     ScopedTiming t(RMM_STEP_SKETCH, stream);
-    return launch_tc<tc::A_GEN, tc::B_MN>(nullptr, X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, status, stream);
+    return launch_sketch(X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, reinterpret_cast<float*>(ws + w.scratch_off),
+                         status, stream);
   }
   if (Y) {
     ScopedTiming t(RMM_STEP_Y, stream);
@@ -261,24 +295,18 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
   if (dt == RMM_DTYPE_BF16) {
     if (dX) {
       ScopedTiming t(RMM_STEP_DX, stream);
-      st = launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, 0, pk, status, stream);
+      st = launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, status, stream);
       if (st != RMM_OK) return st;
     }
     {
+      // db = dY^T 1 comes out of the same contraction as the extra row of ones of S^T
       ScopedTiming t(RMM_STEP_SDY, stream);
-      st = launch_tc<tc::A_GEN, tc::B_MN>(nullptr, dY, G, nullptr, B_proj, D_out, N, c, dist, pk, status, stream);
+      st = launch_sketch(dY, G, db, B_proj, D_out, N, c, dist, pk, reinterpret_cast<float*>(ws + w.scratch_off), status,
+                         stream);
       if (st != RMM_OK) return st;
     }
-    {
-      ScopedTiming t(RMM_STEP_DW, stream);
-      st = launch_tc<tc::A_MN, tc::B_MN>(G, X_proj, dW, nullptr, D_out, D_in, B_proj, 1.0f, 0, pk, status, stream);
-      if (st != RMM_OK) return st;
-    }
-    if (db) {
-      ScopedTiming t(RMM_STEP_DB, stream);
-      return launch_db<__nv_bfloat16>(dY, N, D_out, w, ws, db, stream);
-    }
-    return RMM_OK;
+    ScopedTiming t(RMM_STEP_DW, stream);
+    return launch_tc<tc::A_MN, tc::B_MN>(G, X_proj, dW, nullptr, D_out, D_in, B_proj, 1.0f, status, stream);
   }
   if (dX) {
     ScopedTiming t(RMM_STEP_DX, stream);

@@ -1,24 +1,20 @@
 // Tensor-core contraction kernel for the bf16 mode (sm_100a): C = alpha * A B^T (+ bias),
 // bf16 operands, fp32 accumulation in tensor memory, one 128 x 256 output tile per CTA.
 //
-// The five contractions of Algorithm 1 differ only in where the operands come from:
+// The three dense contractions of Algorithm 1 whose operands all live in memory differ only
+// in the operand layouts (the two sketch contractions are in tc_sketch.cuh):
 //   A_K   : A[m][k] row-major (k contiguous), fetched by TMA           (Y: X,  dX: dY)
 //   A_MN  : A given as [k][m] row-major (m contiguous), fetched by TMA (dW: G = S^T dY)
-//   A_GEN : A[m][k] = P[token k][sketch column m], generated in shared memory by the
-//           CTA's own warps from the Philox seed, never read from memory (X_proj, G)
 //   B_K   : B[n][k] row-major (k contiguous)                           (Y: W)
-//   B_MN  : B given as [k][n] row-major (n contiguous)                 (X_proj: X, dX: W,
-//                                                                       G: dY, dW: X_proj)
+//   B_MN  : B given as [k][n] row-major (n contiguous)                 (dX: W, dW: X_proj)
 // "MN-major" operands are consumed in place through the transpose bits of the tcgen05
 // instruction descriptor; nothing is transposed in memory.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = tensor-memory owner and MMA issuer,
-// warps 2.. = S generators (A_GEN) and epilogue.  Stages of a ring of shared-memory
-// buffers are handed over with mbarriers: full (TMA bytes landed), fullA (generated
-// tile written and fenced to the async proxy), empty (tcgen05.commit: the MMAs that
-// read the stage have retired), accfull (all MMAs of the tile retired).
+// warps 2..5 = epilogue.  Stages of a ring of shared-memory buffers are handed over with
+// mbarriers: full (TMA bytes landed), empty (tcgen05.commit: the MMAs that read the stage
+// have retired), accfull (all MMAs of the tile retired).
 #pragma once
-#include "sketch_rng.cuh"
 #include "tc_common.cuh"
 
 namespace rmm {
@@ -33,7 +29,7 @@ constexpr int SLAB_BYTES = 64 * BK * 2;       // one [64 k][64 mn] MN-major slab
 constexpr int TMEM_COLS = 256;
 constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
-enum : int { A_K = 0, A_MN = 1, A_GEN = 2 };
+enum : int { A_K = 0, A_MN = 1 };
 enum : int { B_K = 0, B_MN = 1 };
 
 struct GemmParams {
@@ -42,7 +38,6 @@ struct GemmParams {
   int64_t ldc;
   const void* bias;   // bf16 [N] or nullptr
   float alpha;
-  int dist;           // A_GEN only: 0 Gaussian, 1 Rademacher, 2 identity
   int* status;        // workspace status word
 };
 
@@ -51,57 +46,20 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// Fill one 128 x 64 K-major, 128-byte-swizzled stage with S^T[m0 .. m0+127][n0 .. n0+63].
-// Row r occupies bytes [128 r, 128 r + 128); its 16-byte chunk c sits at chunk c ^ (r & 7).
-template <int NGEN_THREADS>
-__device__ __forceinline__ void generate_a_stage(uint8_t* a_tile, const PhiloxKey& pk, int dist, int64_t m0,
-                                                 int64_t n0, int gtid) {
-  static_assert(NGEN_THREADS == 256, "task mapping assumes 256 generator threads");
-  if (dist == 0) {
-#pragma unroll 2
-    for (int it = 0; it < 4; ++it) {
-      const int t = it * NGEN_THREADS + gtid;
-      const int r = t >> 3, c = t & 7;
-      const uint4 v = gaussian_8_bf16(pk, (uint32_t)(n0 + 8 * c), (uint32_t)(m0 + r));
-      *reinterpret_cast<uint4*>(a_tile + r * 128 + ((c ^ (r & 7)) << 4)) = v;
-    }
-  } else if (dist == 1) {
-    const int r = gtid >> 1, h = gtid & 1;
-    uint32_t w[4];
-    rademacher_128(pk, (uint32_t)(n0 >> 7), (uint32_t)(m0 + r), w);
-    const uint32_t word = w[((n0 & 127) >> 5) + h];
-#pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int c = 4 * h + b;
-      *reinterpret_cast<uint4*>(a_tile + r * 128 + ((c ^ (r & 7)) << 4)) = rademacher_8_bf16(word, b);
-    }
-  } else {
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-      const int t = it * NGEN_THREADS + gtid;
-      const int r = t >> 3, c = t & 7;
-      const int64_t d = (m0 + r) - (n0 + 8 * c);   // position of the 1 inside this chunk, if any
-      uint32_t q[4] = {0u, 0u, 0u, 0u};
-      if (d >= 0 && d < 8) q[d >> 1] = (d & 1) ? 0x3f800000u : 0x00003f80u;
-      *reinterpret_cast<uint4*>(a_tile + r * 128 + ((c ^ (r & 7)) << 4)) = make_uint4(q[0], q[1], q[2], q[3]);
-    }
-  }
-}
+constexpr int NEPI = 4;   // epilogue warps: one per tensor-memory lane quarter
 
-template <int AMODE, int BMODE, int NEPI>
+template <int AMODE, int BMODE>
 __global__ void __launch_bounds__(64 + 32 * NEPI, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p,
-            PhiloxKey pk) {
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto fulla_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };
-  const uint32_t accfull_bar = bar0 + 8u * (3 * STAGES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * STAGES + 1);
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  const uint32_t accfull_bar = bar0 + 8u * (2 * STAGES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -111,7 +69,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(full_bar(s), 1);
-      mbar_init(fulla_bar(s), 32 * NEPI);
       mbar_init(empty_bar(s), 1);
     }
     mbar_init(accfull_bar, 1);
@@ -130,18 +87,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      if (AMODE != A_GEN) tma_prefetch_desc(&tmA);
+      tma_prefetch_desc(&tmA);
       tma_prefetch_desc(&tmB);
       for (int kb = 0; kb < num_kb; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
         if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) break;
         const uint32_t a_smem = sbase + s * STAGE_BYTES, b_smem = a_smem + A_BYTES;
-        mbar_arrive_expect_tx(full_bar(s), (AMODE != A_GEN ? A_BYTES : 0) + B_BYTES);
+        mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES);
         const int k0 = kb * BK;
         if (AMODE == A_K) {
           tma_load_2d(a_smem, &tmA, full_bar(s), k0, (int)m0);
-        } else if (AMODE == A_MN) {
+        } else {
 #pragma unroll
           for (int sl = 0; sl < BM / 64; ++sl) tma_load_2d(a_smem + sl * SLAB_BYTES, &tmA, full_bar(s), (int)m0 + 64 * sl, k0);
         }
@@ -163,7 +120,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int s = kb % STAGES;
         const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
         ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
-        if (ok && AMODE == A_GEN) ok = mbar_wait(fulla_bar(s), ph, abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t a_smem = sbase + s * STAGE_BYTES, b_smem = a_smem + A_BYTES;
@@ -181,30 +137,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ generators + epilogue
-    const int ew = warp - 2;
-    if constexpr (AMODE == A_GEN) {
-      const int gtid = threadIdx.x - 64;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) break;
-        generate_a_stage<32 * NEPI>(smem + s * STAGE_BYTES, pk, p.dist, m0, (int64_t)kb * BK, gtid);
-        fence_proxy_async_smem();
-        mbar_arrive(fulla_bar(s));
-      }
-    }
+    // ------------------------------------------------------------ epilogue
     const bool acc_ready = __all_sync(0xffffffffu, mbar_wait(accfull_bar, 0u, abort_flag, p.status));
     if (acc_ready) {
       tc_fence_after();
       const int q = warp & 3;                       // tensor-memory lane quarter this warp may read
-      constexpr int CHUNKS = (BN / 32) / (NEPI / 4);
-      const int c_begin = (ew >> 2) * CHUNKS;
+      constexpr int CHUNKS = BN / 32;
       const int64_t row = m0 + q * 32 + lane;
       __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc;
       const __nv_bfloat16* bias = reinterpret_cast<const __nv_bfloat16*>(p.bias);
       for (int cc = 0; cc < CHUNKS; ++cc) {
-        const int c = c_begin + cc;
+        const int c = cc;
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
         tmem_ld_wait();

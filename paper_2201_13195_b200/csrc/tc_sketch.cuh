@@ -1,0 +1,341 @@
+// Sketch contraction on the tensor cores (bf16 mode, sm_100a):
+//     C[j][d] = sum over tokens n of P[n][j] * B[n][d]
+// i.e. X_proj = S^T X in the forward pass and G = S^T dY in the backward pass of
+// Algorithm 1, with the 128 x 64 tiles of S^T generated in shared memory from the Philox
+// seed by the CTA's own warps (S is never read from or written to memory) and B (X or
+// dY, row-major [tokens][d]) streamed by TMA as an MN-major operand.
+//
+// Work decomposition.  An output tile is 128 sketch rows x 512 columns: the whole tensor
+// memory of an SM (512 fp32 columns) accumulates it, so that every generated entry of S
+// is used 512 times.  There are far fewer such tiles than SMs and each has a long
+// contraction (all tokens), so the (tile, 64-token step) units are laid out in one line
+// and cut into equal contiguous ranges, one per CTA.  A CTA accumulates each of the (at
+// most a few) tile segments in its range in tensor memory and writes it as an fp32
+// partial tile; sketch_reduce_kernel adds the partial tiles of every output tile in a
+// fixed order, applies the scale c = 1/sqrt(B_proj) (Eq. 5) and rounds to bf16.
+//
+// db for free: when ones_row is set, row index B_proj of S^T is a row of ones, so row
+// B_proj of the result is sum_n dY[n][:] (Eq. 3); the reduce kernel stores it, unscaled.
+//
+// Warp roles: warp 0 TMA producer (B), warp 1 tensor-memory owner and MMA issuer, warps
+// 2..17 generate S tiles and drain the accumulator.  A stages hold 64 tokens, B stages 32
+// tokens (so that four of each fit in shared memory); all waits are bounded.
+#pragma once
+#include "sketch_rng.cuh"
+#include "tc_common.cuh"
+
+namespace rmm {
+namespace tc {
+
+constexpr int SK_BM = 128, SK_BN = 512, SK_AK = 64, SK_BK = 32;
+constexpr int SK_A_STAGES = 4, SK_B_STAGES = 4;
+constexpr int SK_A_BYTES = SK_BM * SK_AK * 2;        // 16 KiB
+constexpr int SK_B_BYTES = SK_BN * SK_BK * 2;        // 32 KiB
+constexpr int SK_B_SLAB = 64 * SK_BK * 2;            // [32 tokens][64 columns] = 4 KiB
+constexpr int SK_GEN_WARPS = 16;
+constexpr int SK_GEN_THREADS = 32 * SK_GEN_WARPS;
+constexpr int SK_THREADS = 64 + SK_GEN_THREADS;
+constexpr int SK_SMEM_BYTES = SK_A_STAGES * SK_A_BYTES + SK_B_STAGES * SK_B_BYTES + 1024 + 256;
+constexpr int SK_TILE_ELEMS = SK_BM * SK_BN;         // fp32 elements of one partial tile
+constexpr int SK_MAX_CTAS = 148;                     // grid size used for workspace sizing
+
+// Static schedule shared by the sketch kernel, the reduce kernel and the host.
+struct SketchSchedule {
+  int tiles_m, tiles_n, ksteps;       // output tiles and 64-token steps per tile
+  int num_ctas;
+  long long total_units, units_per_cta, lcm_units;   // lcm(units_per_cta, ksteps)
+  __host__ __device__ long long slot_of(int cta, int tile, long long seg_start) const {
+    // Segments are numbered in unit order; one starts at every CTA-range start and at
+    // every tile start (a unit that is both counts once).
+    return (long long)cta + tile - seg_start / lcm_units;
+  }
+  __host__ __device__ long long num_slots() const { return (long long)num_ctas + (long long)tiles_m * tiles_n; }
+};
+
+inline long long gcd_ll(long long a, long long b) { while (b) { long long t = a % b; a = b; b = t; } return a; }
+
+inline SketchSchedule make_sketch_schedule(long long rows, long long cols, long long tokens, int max_ctas) {
+  SketchSchedule s;
+  s.tiles_m = (int)((rows + SK_BM - 1) / SK_BM);
+  s.tiles_n = (int)((cols + SK_BN - 1) / SK_BN);
+  s.ksteps = (int)((tokens + SK_AK - 1) / SK_AK);
+  s.total_units = (long long)s.tiles_m * s.tiles_n * s.ksteps;
+  s.num_ctas = (int)(s.total_units < max_ctas ? s.total_units : max_ctas);
+  s.units_per_cta = (s.total_units + s.num_ctas - 1) / s.num_ctas;
+  s.num_ctas = (int)((s.total_units + s.units_per_cta - 1) / s.units_per_cta);
+  s.lcm_units = s.units_per_cta / gcd_ll(s.units_per_cta, s.ksteps) * s.ksteps;
+  return s;
+}
+
+struct SketchParams {
+  long long rows;      // rows of S^T that are computed: B_proj (+1 with the ones row)
+  long long b_proj;    // index of the ones row when ones_row != 0
+  long long cols;      // columns of B and of the result
+  long long tokens;    // contraction length
+  float* partial;      // [num_slots][128][512] fp32
+  int dist;
+  int ones_row;
+  int* status;
+  SketchSchedule sched;
+};
+
+// One 128 x 64 stage of S^T, K-major with the 128-byte swizzle: row r at byte 128 r, its
+// 16-byte chunk c (tokens 8c .. 8c+7) stored at chunk position c ^ (r & 7).
+__device__ __forceinline__ void sketch_generate_stage(uint8_t* a_tile, const PhiloxKey& pk, const SketchParams& p,
+                                                      long long m0, long long n0, int gtid) {
+  constexpr uint32_t kOnes = 0x3f803f80u;   // two bf16 1.0
+  if (p.dist == 0) {
+#pragma unroll
+    for (int it = 0; it < (SK_BM * 8) / SK_GEN_THREADS; ++it) {
+      const int t = it * SK_GEN_THREADS + gtid;
+      const int r = t >> 3, c = t & 7;
+      uint4 v = gaussian_8_bf16(pk, (uint32_t)(n0 + 8 * c), (uint32_t)(m0 + r));
+      if (p.ones_row && m0 + r == p.b_proj) v = make_uint4(kOnes, kOnes, kOnes, kOnes);
+      *reinterpret_cast<uint4*>(a_tile + r * 128 + ((c ^ (r & 7)) << 4)) = v;
+    }
+  } else if (p.dist == 1) {
+    // one thread per (row, 16 tokens): 2 chunks out of one Philox word
+    const int r = gtid >> 2, h = gtid & 3;
+    uint32_t w[4];
+    rademacher_128(pk, (uint32_t)(n0 >> 7), (uint32_t)(m0 + r), w);
+    const uint32_t word = w[((n0 & 127) >> 5) + (h >> 1)];
+    const bool ones = p.ones_row && m0 + r == p.b_proj;
+#pragma unroll
+    for (int b = 0; b < 2; ++b) {
+      const int c = 2 * h + b;
+      uint4 v = rademacher_8_bf16(word, 2 * (h & 1) + b);
+      if (ones) v = make_uint4(kOnes, kOnes, kOnes, kOnes);
+      *reinterpret_cast<uint4*>(a_tile + r * 128 + ((c ^ (r & 7)) << 4)) = v;
+    }
+  } else {
+#pragma unroll
+    for (int it = 0; it < (SK_BM * 8) / SK_GEN_THREADS; ++it) {
+      const int t = it * SK_GEN_THREADS + gtid;
+      const int r = t >> 3, c = t & 7;
+      const long long d = (m0 + r) - (n0 + 8 * c);
+      uint32_t q0 = 0, q1 = 0, q2 = 0, q3 = 0;
+      if (d >= 0 && d < 8) {
+        const uint32_t one = (d & 1) ? 0x3f800000u : 0x00003f80u;
+        const int wi = (int)(d >> 1);
+        q0 = wi == 0 ? one : 0u; q1 = wi == 1 ? one : 0u; q2 = wi == 2 ? one : 0u; q3 = wi == 3 ? one : 0u;
+      }
+      uint4 v = make_uint4(q0, q1, q2, q3);
+      if (p.ones_row && m0 + r == p.b_proj) v = make_uint4(kOnes, kOnes, kOnes, kOnes);
+      *reinterpret_cast<uint4*>(a_tile + r * 128 + ((c ^ (r & 7)) << 4)) = v;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(SK_THREADS, 1)
+sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey pk) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* a_ring = smem;
+  uint8_t* b_ring = smem + SK_A_STAGES * SK_A_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(b_ring + SK_B_STAGES * SK_B_BYTES);
+  const uint32_t bar0 = smem_u32(bars);
+  auto fulla_bar = [&](int s) { return bar0 + 8u * s; };
+  auto emptya_bar = [&](int s) { return bar0 + 8u * (SK_A_STAGES + s); };
+  auto fullb_bar = [&](int s) { return bar0 + 8u * (2 * SK_A_STAGES + s); };
+  auto emptyb_bar = [&](int s) { return bar0 + 8u * (2 * SK_A_STAGES + SK_B_STAGES + s); };
+  const uint32_t accfull_bar = bar0 + 8u * (2 * SK_A_STAGES + 2 * SK_B_STAGES);
+  const uint32_t accempty_bar = accfull_bar + 8u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * SK_A_STAGES + 2 * SK_B_STAGES + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const SketchSchedule& sc = p.sched;
+  const long long u_begin = (long long)blockIdx.x * sc.units_per_cta;
+  const long long u_end = (u_begin + sc.units_per_cta < sc.total_units) ? u_begin + sc.units_per_cta : sc.total_units;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < SK_A_STAGES; ++s) {
+      mbar_init(fulla_bar(s), SK_GEN_THREADS);
+      mbar_init(emptya_bar(s), 1);
+    }
+    for (int s = 0; s < SK_B_STAGES; ++s) {
+      mbar_init(fullb_bar(s), 1);
+      mbar_init(emptyb_bar(s), 1);
+    }
+    mbar_init(accfull_bar, 1);
+    mbar_init(accempty_bar, SK_GEN_THREADS);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (B)
+    if (lane == 0) {
+      tma_prefetch_desc(&tmB);
+      long long it = 0;   // running 32-token stage counter
+      bool ok = true;
+      for (long long u = u_begin; u < u_end && ok;) {
+        const int tile = (int)(u / sc.ksteps);
+        const int ks0 = (int)(u % sc.ksteps);
+        const long long rem = u_end - u;
+        const int ks1 = (int)((sc.ksteps - ks0 < rem) ? sc.ksteps : ks0 + rem);
+        const int n0 = (tile % sc.tiles_n) * SK_BN;
+        for (int ks = ks0; ks < ks1 && ok; ++ks) {
+          for (int half = 0; half < 2; ++half, ++it) {
+            const int s = (int)(it % SK_B_STAGES);
+            const uint32_t ph = (uint32_t)(it / SK_B_STAGES) & 1u;
+            if (!mbar_wait(emptyb_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t b_smem = smem_u32(b_ring + s * SK_B_BYTES);
+            mbar_arrive_expect_tx(fullb_bar(s), SK_B_BYTES);
+            const int tok0 = ks * SK_AK + half * SK_BK;
+#pragma unroll
+            for (int sl = 0; sl < SK_BN / 64; ++sl)
+              tma_load_2d(b_smem + sl * SK_B_SLAB, &tmB, fullb_bar(s), n0 + 64 * sl, tok0);
+          }
+        }
+        u += ks1 - ks0;
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16(SK_BM, 256, false, true);
+      long long ita = 0, itb = 0;
+      int seg = 0;
+      bool ok = true;
+      for (long long u = u_begin; u < u_end && ok; ++seg) {
+        const int ks0 = (int)(u % sc.ksteps);
+        const long long rem = u_end - u;
+        const int ks1 = (int)((sc.ksteps - ks0 < rem) ? sc.ksteps : ks0 + rem);
+        if (seg > 0) {   // the previous segment's accumulator must have been drained
+          ok = mbar_wait(accempty_bar, (uint32_t)(seg - 1) & 1u, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        for (int ks = ks0; ks < ks1 && ok; ++ks, ++ita) {
+          const int sa = (int)(ita % SK_A_STAGES);
+          ok = mbar_wait(fulla_bar(sa), (uint32_t)(ita / SK_A_STAGES) & 1u, abort_flag, p.status);
+          if (!ok) break;
+          const uint32_t a_smem = smem_u32(a_ring + sa * SK_A_BYTES);
+          for (int half = 0; half < 2; ++half, ++itb) {
+            const int sb = (int)(itb % SK_B_STAGES);
+            ok = mbar_wait(fullb_bar(sb), (uint32_t)(itb / SK_B_STAGES) & 1u, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t b_smem = smem_u32(b_ring + sb * SK_B_BYTES);
+#pragma unroll
+            for (int j = 0; j < SK_BK / 16; ++j) {
+              const uint64_t adesc = smem_desc_sw128(a_smem + (half * (SK_BK / 16) + j) * 32, 16, 1024);
+#pragma unroll
+              for (int nh = 0; nh < 2; ++nh) {
+                const uint64_t bdesc = smem_desc_sw128(b_smem + nh * 4 * SK_B_SLAB + j * 2048, SK_B_SLAB, 1024);
+                umma_bf16(tmem_base + nh * 256, adesc, bdesc, idesc, (ks > ks0 || half > 0 || j > 0) ? 1u : 0u);
+              }
+            }
+            umma_commit(emptyb_bar(sb));
+          }
+          if (ok) umma_commit(emptya_bar(sa));
+        }
+        if (ok) umma_commit(accfull_bar);
+        u += ks1 - ks0;
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ S generators + accumulator drain
+    const int gtid = threadIdx.x - 64;
+    const int gw = warp - 2;
+    long long ita = 0;
+    int seg = 0;
+    bool ok = true;
+    for (long long u = u_begin; u < u_end && ok; ++seg) {
+      const int tile = (int)(u / sc.ksteps);
+      const int ks0 = (int)(u % sc.ksteps);
+      const long long rem = u_end - u;
+      const int ks1 = (int)((sc.ksteps - ks0 < rem) ? sc.ksteps : ks0 + rem);
+      const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
+      for (int ks = ks0; ks < ks1; ++ks, ++ita) {
+        const int sa = (int)(ita % SK_A_STAGES);
+        if (!mbar_wait(emptya_bar(sa), ((uint32_t)(ita / SK_A_STAGES) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        sketch_generate_stage(a_ring + sa * SK_A_BYTES, pk, p, m0, (long long)ks * SK_AK, gtid);
+        fence_proxy_async_smem();
+        mbar_arrive(fulla_bar(sa));
+      }
+      ok = __all_sync(0xffffffffu, ok && mbar_wait(accfull_bar, (uint32_t)seg & 1u, abort_flag, p.status));
+      if (!ok) break;
+      tc_fence_after();
+      {
+        const int q = warp & 3;                 // tensor-memory lane quarter of this warp
+        const int cgroup = gw >> 2;             // 4 warps share a quarter: 128 columns each
+        const long long seg_start = u;
+        float* slot = p.partial + sc.slot_of((int)blockIdx.x, tile, seg_start) * (long long)SK_TILE_ELEMS;
+        float* prow = slot + (long long)(q * 32 + lane) * SK_BN;
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c = cgroup * 4 + cc;
+          uint32_t v[32];
+          tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            *reinterpret_cast<uint4*>(prow + c * 32 + g * 4) = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(accempty_bar);
+      u += ks1 - ks0;
+    }
+  }
+  // ---------------------------------------------------------------- teardown
+  if (*abort_flag) {
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 1000000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+// Adds the partial tiles of each output tile in schedule order, scales, rounds to bf16.
+// grid = (tiles, 128 / SKR_ROWS), block = 128 threads: thread t owns columns 4t .. 4t+3.
+constexpr int SKR_ROWS = 8;
+__global__ void __launch_bounds__(128)
+sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ ones_out) {
+  const SketchSchedule& sc = p.sched;
+  const int tile = blockIdx.x;
+  const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM, n0 = (long long)(tile % sc.tiles_n) * SK_BN;
+  const long long t_begin = (long long)tile * sc.ksteps, t_end = t_begin + sc.ksteps;
+  const int c_first = (int)(t_begin / sc.units_per_cta), c_last = (int)((t_end - 1) / sc.units_per_cta);
+  const int col = threadIdx.x * 4;
+  if (n0 + col >= p.cols) return;
+  for (int rr = 0; rr < SKR_ROWS; ++rr) {
+    const int r = blockIdx.y * SKR_ROWS + rr;
+    const long long j = m0 + r;
+    if (j >= p.rows) break;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = c_first; c <= c_last; ++c) {
+      const long long cs = (long long)c * sc.units_per_cta;
+      const long long seg_start = cs > t_begin ? cs : t_begin;
+      const float* slot = p.partial + sc.slot_of(c, tile, seg_start) * (long long)SK_TILE_ELEMS;
+      const float4 v = *reinterpret_cast<const float4*>(slot + (long long)r * SK_BN + col);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    const bool is_ones = p.ones_row && j == p.b_proj;
+    const float s = is_ones ? 1.0f : scale;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * s, acc.y * s), hi = __floats2bfloat162_rn(acc.z * s, acc.w * s);
+    uint2 o = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+    // cols is a multiple of 8 and col a multiple of 4: the 4 columns are all inside or all outside
+    if (is_ones) {
+      if (ones_out) *reinterpret_cast<uint2*>(ones_out + n0 + col) = o;
+    } else {
+      *reinterpret_cast<uint2*>(out + j * p.cols + n0 + col) = o;
+    }
+  }
+}
+
+}  // namespace tc
+}  // namespace rmm
