@@ -146,6 +146,33 @@ rmm_status rmm_profile_enable(int capacity);
 int rmm_profile_read(int* step_ids, float* milliseconds, int max_records);
 
 /*
+ * Bias gradient without any allocation (the paper has no counterpart; it computes the
+ * same db = dY^T 1 of Eq. 3 that rmm_backward returns).
+ *
+ * For callers that hold no workspace and cannot obtain one: code running inside a
+ * memory-pool or graph-replay region where cudaMalloc (and with it every allocating
+ * library routine, PyTorch's caching allocator included) is forbidden, or late in a
+ * step when the device is full.  rmm_backward needs caller-provided scratch for its
+ * partial sums; this entry point keeps that scratch in a fixed array that is part of
+ * the library image: RMM_BIAS_GRAD_STATIC_SLICES x RMM_BIAS_GRAD_STATIC_MAX_D_OUT
+ * fp32 values = 256 KiB, resident on every GPU that loads the library until the process
+ * exits.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *   in : dY [N, D_out] (device, row-major, 16-byte aligned), dt = element type
+ *   out: db [D_out] (device) = column sums of dY, accumulated in fp32
+ * Returns RMM_ERR_UNSUPPORTED when D_out > RMM_BIAS_GRAD_STATIC_MAX_D_OUT, and
+ * RMM_ERR_INVALID_ARG for null or misaligned pointers or non-positive sizes.
+ * The first call on each device looks up the device address of the array (one driver
+ * query, with that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's partial
+ * sums: every value that is read is rewritten first, so nothing needs clearing, but two
+ * calls that may run concurrently on the same device (different streams) race on it.
+ */
+#define RMM_BIAS_GRAD_STATIC_MAX_D_OUT 4096
+#define RMM_BIAS_GRAD_STATIC_SLICES 16
+rmm_status rmm_bias_grad_static(const void* dY, int64_t N, int64_t D_out, rmm_dtype dt, void* db,
+                                void* cuda_stream);
+
+/*
  * Host-buffer convenience wrappers (end-to-end path): the tensor arguments are HOST
  * pointers (pinned memory recommended); the device buffers dev_* and the workspace
  * are caller-owned DEVICE scratch of at least the tensors' sizes.  Each call copies

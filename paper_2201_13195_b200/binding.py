@@ -18,7 +18,9 @@ RMM_DTYPE_BF16, RMM_DTYPE_F32 = 0, 1
 
 EXPORTS = ("rmm_workspace_bytes", "rmm_forward", "rmm_backward", "rmm_debug_generate_s",
            "rmm_last_device_status", "rmm_status_string", "rmm_host_staging_bytes",
-           "rmm_forward_host", "rmm_backward_host", "rmm_profile_enable", "rmm_profile_read")
+           "rmm_forward_host", "rmm_backward_host", "rmm_profile_enable", "rmm_profile_read",
+           "rmm_bias_grad_static")
+RMM_BIAS_GRAD_STATIC_MAX_D_OUT = 4096
 STEP_NAMES = ("y", "sketch", "dx", "sdy", "dw", "db")
 
 if not os.path.exists(LIB_PATH):
@@ -45,6 +47,8 @@ _lib.rmm_forward_host.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _
 _lib.rmm_forward_host.restype = _int
 _lib.rmm_backward_host.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.rmm_backward_host.restype = _int
+_lib.rmm_bias_grad_static.argtypes = [_vp, _i64, _i64, _int, _vp, _vp]
+_lib.rmm_bias_grad_static.restype = _int
 _lib.rmm_profile_enable.argtypes = [_int]
 _lib.rmm_profile_enable.restype = _int
 _lib.rmm_profile_read.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_float), _int]
@@ -181,3 +185,17 @@ def rmm_profile_read(max_records: int):
     ms = (C.c_float * max_records)()
     n = _lib.rmm_profile_read(ids, ms, max_records)
     return [(STEP_NAMES[ids[i]], float(ms[i])) for i in range(n)]
+
+
+def rmm_bias_grad_static(dY, db=None, stream=None):
+    """db = column sums of dY through the entry point that allocates nothing in the library
+    (its scratch is a fixed array inside librmm.so).  Pass `db` to avoid the one output
+    allocation this wrapper would otherwise make; D_out is limited to
+    RMM_BIAS_GRAD_STATIC_MAX_D_OUT."""
+    N, D_out = dY.shape
+    assert dY.is_cuda and dY.is_contiguous()
+    if db is None:
+        db = torch.empty((D_out,), dtype=dY.dtype, device=dY.device)
+    _check(_lib.rmm_bias_grad_static(_ptr(dY), N, D_out, _dtype_code(dY), _ptr(db), _stream_ptr(stream)),
+           "rmm_bias_grad_static")
+    return db

@@ -208,6 +208,30 @@ rmm_status launch_db(const void* dY, int64_t N, int64_t D_out, const Workspace& 
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
 
+// ------------------------------------------------------------------ allocation-free bias gradient
+// Scratch for rmm_bias_grad_static: partial column sums, [slice][column].  The name below
+// is only a host-side handle; kernels get the device address from cudaGetSymbolAddress.
+static __device__ __align__(256) float g_bias_grad_scratch[RMM_BIAS_GRAD_STATIC_SLICES * RMM_BIAS_GRAD_STATIC_MAX_D_OUT];
+
+constexpr int kMaxDevices = 64;
+float* g_bias_grad_scratch_addr[kMaxDevices] = {};
+std::mutex g_bias_grad_mutex;
+
+// Device address of the scratch array on the current device (looked up once per device).
+rmm_status bias_grad_scratch(float** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RMM_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_bias_grad_mutex);
+  if (g_bias_grad_scratch_addr[dev] == nullptr) {
+    float* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_bias_grad_scratch) != cudaSuccess || ptr == nullptr)
+      return RMM_ERR_CUDA;
+    g_bias_grad_scratch_addr[dev] = ptr;
+  }
+  *out = g_bias_grad_scratch_addr[dev];
+  return RMM_OK;
+}
+
 // ------------------------------------------------------------------ argument checks
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -366,6 +390,34 @@ const char* rmm_status_string(rmm_status s) {
     case RMM_ERR_TIMEOUT: return "RMM_ERR_TIMEOUT";
   }
   return "RMM_ERR_UNKNOWN";
+}
+
+rmm_status rmm_bias_grad_static(const void* dY, int64_t N, int64_t D_out, rmm_dtype dt, void* db, void* cuda_stream) {
+  if (!dY || !db || N < 1 || D_out < 1) return RMM_ERR_INVALID_ARG;
+  if (dt != RMM_DTYPE_BF16 && dt != RMM_DTYPE_F32) return RMM_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(db)) return RMM_ERR_INVALID_ARG;
+  if (D_out > RMM_BIAS_GRAD_STATIC_MAX_D_OUT) return RMM_ERR_UNSUPPORTED;  // would not fit the fixed scratch
+  if (!device_state().ok) return RMM_ERR_CUDA;
+  float* scratch = nullptr;
+  rmm_status st = bias_grad_scratch(&scratch);
+  if (st != RMM_OK) return st;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const int slices = (int)(N < RMM_BIAS_GRAD_STATIC_SLICES ? N : RMM_BIAS_GRAD_STATIC_SLICES);
+  const int rows_per_slice = (int)((N + slices - 1) / slices);
+  const int used = (int)((N + rows_per_slice - 1) / rows_per_slice);
+  dim3 grid((unsigned)((D_out + 255) / 256), (unsigned)used);
+  const unsigned fin_blocks = (unsigned)((D_out + 255) / 256);
+  if (dt == RMM_DTYPE_BF16) {
+    db_partial_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(dY), N, D_out,
+                                                                rows_per_slice, scratch);
+    db_finish_kernel<__nv_bfloat16><<<fin_blocks, 256, 0, stream>>>(scratch, used, D_out,
+                                                                     reinterpret_cast<__nv_bfloat16*>(db));
+  } else {
+    db_partial_kernel<float><<<grid, 256, 0, stream>>>(reinterpret_cast<const float*>(dY), N, D_out, rows_per_slice,
+                                                        scratch);
+    db_finish_kernel<float><<<fin_blocks, 256, 0, stream>>>(scratch, used, D_out, reinterpret_cast<float*>(db));
+  }
+  return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
 
 rmm_status rmm_profile_enable(int capacity) {
