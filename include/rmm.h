@@ -113,6 +113,27 @@ rmm_status rmm_debug_generate_s(uint64_t seed, int64_t N, int64_t B_proj, rmm_di
                                 void* S_out, void* cuda_stream);
 
 /*
+ * Applies the uniform -> normal map of RMM_DIST_GAUSSIAN to n given Philox output words
+ * (device array): out[2i] and out[2i+1] (device, fp32) are the two normals that word i
+ * yields, before any storage rounding.  Debug aid like rmm_debug_generate_s: lets a test
+ * sweep all 2^16 radius inputs and all 2^16 angle inputs of the transform.
+ */
+rmm_status rmm_debug_gauss_words(const uint32_t* words, int64_t n, float* out, void* cuda_stream);
+
+/*
+ * Host-only testing aid (no device needed): the static work schedule of the sketch kernels
+ * for a result of `rows` x `cols` contracted over `tokens`, on `max_ctas` CTAs.
+ *   mode 0: one record (cta, tile, first step, end step, slot) per work segment, in the
+ *           order in which each CTA executes them;
+ *   mode 1: one record (tile, slot, 0, 0, 0) per partial tile in the order in which the
+ *           reduction adds them.
+ * Writes at most `cap` records of five int64 to `records` (host memory) and returns the
+ * number of records that exist; info[0..3] = tiles, 64-token steps per tile, grid size, slots.
+ */
+int64_t rmm_debug_sketch_schedule(int64_t rows, int64_t cols, int64_t tokens, int max_ctas, int mode,
+                                  int64_t* records, int64_t cap, int64_t* info);
+
+/*
  * Reads the status word that the kernels of the last call using this workspace left
  * there.  HOST-synchronous on the device-to-host copy of one word: the caller must
  * have synchronised the stream first.  Returns RMM_OK or RMM_ERR_TIMEOUT (or

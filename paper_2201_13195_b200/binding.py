@@ -19,7 +19,7 @@ RMM_DTYPE_BF16, RMM_DTYPE_F32 = 0, 1
 EXPORTS = ("rmm_workspace_bytes", "rmm_forward", "rmm_backward", "rmm_debug_generate_s",
            "rmm_last_device_status", "rmm_status_string", "rmm_host_staging_bytes",
            "rmm_forward_host", "rmm_backward_host", "rmm_profile_enable", "rmm_profile_read",
-           "rmm_bias_grad_static")
+           "rmm_bias_grad_static", "rmm_debug_gauss_words", "rmm_debug_sketch_schedule")
 RMM_BIAS_GRAD_STATIC_MAX_D_OUT = 4096
 STEP_NAMES = ("y", "sketch", "dx", "sdy", "dw", "db")
 
@@ -49,6 +49,10 @@ _lib.rmm_backward_host.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, 
 _lib.rmm_backward_host.restype = _int
 _lib.rmm_bias_grad_static.argtypes = [_vp, _i64, _i64, _int, _vp, _vp]
 _lib.rmm_bias_grad_static.restype = _int
+_lib.rmm_debug_gauss_words.argtypes = [_vp, _i64, _vp, _vp]
+_lib.rmm_debug_gauss_words.restype = _int
+_lib.rmm_debug_sketch_schedule.argtypes = [_i64, _i64, _i64, _int, _int, _vp, _i64, _vp]
+_lib.rmm_debug_sketch_schedule.restype = _i64
 _lib.rmm_profile_enable.argtypes = [_int]
 _lib.rmm_profile_enable.restype = _int
 _lib.rmm_profile_read.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_float), _int]
@@ -199,3 +203,23 @@ def rmm_bias_grad_static(dY, db=None, stream=None):
     _check(_lib.rmm_bias_grad_static(_ptr(dY), N, D_out, _dtype_code(dY), _ptr(db), _stream_ptr(stream)),
            "rmm_bias_grad_static")
     return db
+
+
+def rmm_debug_gauss_words(words, stream=None):
+    """fp32 [n, 2]: the (even, odd) normals the Gaussian transform makes of each uint32 word
+    (words: device tensor of n bit patterns stored as int32)."""
+    assert words.is_cuda and words.dtype == torch.int32 and words.is_contiguous()
+    out = torch.empty((words.numel(), 2), dtype=torch.float32, device=words.device)
+    _check(_lib.rmm_debug_gauss_words(_ptr(words), words.numel(), _ptr(out), _stream_ptr(stream)),
+           "rmm_debug_gauss_words")
+    return out
+
+
+def rmm_debug_sketch_schedule(rows, cols, tokens, max_ctas=148, mode=0):
+    """(records, info): the sketch kernels' static schedule as lists of 5-tuples (host only)."""
+    info = (C.c_int64 * 4)()
+    n = _lib.rmm_debug_sketch_schedule(rows, cols, tokens, max_ctas, mode, None, 0, C.addressof(info))
+    buf = (C.c_int64 * (5 * max(n, 1)))()
+    _lib.rmm_debug_sketch_schedule(rows, cols, tokens, max_ctas, mode, C.addressof(buf), n, C.addressof(info))
+    recs = [tuple(buf[5 * i + j] for j in range(5)) for i in range(n)]
+    return recs, {"tiles": info[0], "ksteps": info[1], "num_ctas": info[2], "num_slots": info[3]}

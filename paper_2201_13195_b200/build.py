@@ -24,7 +24,7 @@ def _newest_source_mtime() -> float:
 def nvcc_command(out: str, extra=()):
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     return [nvcc, "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
-            "-Xcompiler", "-fPIC", "-shared", "--fmad=true", "-o", out,
+            "-Xcompiler", "-fPIC", "-shared", "--fmad=true", "--extended-lambda", "-diag-suppress", "20013,20015", "-o", out,
             *[os.path.join(CSRC, s) for s in SOURCES], *extra]
 
 

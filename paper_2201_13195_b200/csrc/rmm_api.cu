@@ -150,7 +150,7 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   tc::GemmParams p;
   p.M = M; p.N = N; p.K = K;
   p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.status = status;
-  dim3 grid((unsigned)((M + tc::BM - 1) / tc::BM), (unsigned)((N + tc::BN - 1) / tc::BN));
+  dim3 grid((unsigned)((N + tc::BN - 1) / tc::BN), (unsigned)((M + tc::BM - 1) / tc::BM));
   tc::gemm_kernel<AMODE, BMODE><<<grid, 64 + 32 * tc::NEPI, tc::GEMM_SMEM_BYTES, stream>>>(tmA, tmB, p);
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
@@ -173,7 +173,7 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   const int sms = device_state().num_sms;
   p.sched = tc::make_sketch_schedule(p.rows, cols, tokens, sms < tc::SK_MAX_CTAS ? sms : tc::SK_MAX_CTAS);
   tc::sketch_kernel<<<p.sched.num_ctas, tc::SK_THREADS, tc::SK_SMEM_BYTES, stream>>>(tmB, p, pk);
-  dim3 rgrid((unsigned)(p.sched.tiles_m * p.sched.tiles_n), tc::SK_BM / tc::SKR_ROWS);
+  dim3 rgrid((unsigned)p.sched.tiles(), tc::SK_BM / tc::SKR_ROWS);
   tc::sketch_reduce_kernel<<<rgrid, 128, 0, stream>>>(p, c, reinterpret_cast<__nv_bfloat16*>(out),
                                                       reinterpret_cast<__nv_bfloat16*>(ones_out));
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
@@ -371,6 +371,43 @@ rmm_status rmm_debug_generate_s(uint64_t seed, int64_t N, int64_t B_proj, rmm_di
   else
     dump_sketch_kernel<float><<<blocks, 256, 0, stream>>>(pk, (int)dist, N, B_proj, reinterpret_cast<float*>(S_out));
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+
+rmm_status rmm_debug_gauss_words(const uint32_t* words, int64_t n, float* out, void* cuda_stream) {
+  if (!words || !out || n < 1) return RMM_ERR_INVALID_ARG;
+  if (!device_state().ok) return RMM_ERR_CUDA;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  gauss_words_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(words, n, out);
+  return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+
+int64_t rmm_debug_sketch_schedule(int64_t rows, int64_t cols, int64_t tokens, int max_ctas, int mode, int64_t* records,
+                                  int64_t cap, int64_t* info) {
+  if (rows < 1 || cols < 1 || tokens < 1 || max_ctas < 1) return -1;
+  const tc::SketchSchedule sc = tc::make_sketch_schedule(rows, cols, tokens, max_ctas);
+  if (info) {
+    info[0] = sc.tiles(); info[1] = sc.ksteps; info[2] = sc.num_ctas; info[3] = sc.num_slots();
+  }
+  int64_t n = 0;
+  auto put = [&](int64_t a, int64_t b, int64_t c, int64_t d, int64_t e) {
+    if (records && n < cap) {
+      int64_t* r = records + 5 * n;
+      r[0] = a; r[1] = b; r[2] = c; r[3] = d; r[4] = e;
+    }
+    ++n;
+  };
+  if (mode == 0) {
+    for (int cta = 0; cta < sc.num_ctas; ++cta) {
+      int it = 0;
+      long long cursor = 0;
+      tc::SketchSegment sg;
+      while (tc::sketch_next_segment(sc, cta, it, cursor, sg)) put(cta, sg.tile, sg.ks0, sg.ks1, sg.slot);
+    }
+  } else {
+    for (int tile = 0; tile < sc.tiles(); ++tile)
+      tc::sketch_for_each_slot_of_tile(sc, tile, [&](long long slot) { put(tile, slot, 0, 0, 0); });
+  }
+  return n;
 }
 
 rmm_status rmm_last_device_status(const void* workspace) {

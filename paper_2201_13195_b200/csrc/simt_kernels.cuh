@@ -158,4 +158,14 @@ __global__ void dump_sketch_kernel(PhiloxKey pk, int dist, int64_t N, int64_t k,
   out[idx] = from_f32<T>(sketch_entry(pk, dist, n, j, sizeof(T) == 2));
 }
 
+// The normal transform applied to caller-given words (debug entry point).
+__global__ void gauss_words_kernel(const uint32_t* __restrict__ words, int64_t n, float* __restrict__ out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float a, b;
+  gauss_pair(words[i], a, b);
+  out[2 * i] = a;
+  out[2 * i + 1] = b;
+}
+
 }  // namespace rmm

@@ -16,8 +16,8 @@ namespace rmm {
 namespace tc {
 
 constexpr int kStatusTimeout = 5;                 // == RMM_ERR_TIMEOUT
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
-constexpr uint32_t kWaitLimitPolls = 1u << 28;
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM clock per wait
+constexpr uint32_t kWaitLimitPolls = 1u << 30;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -57,15 +57,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false if the abort flag was raised by someone else or if the
-// limit ran out (then it raises the flag itself and records the timeout).
+// limit ran out (then it raises the flag itself and records the timeout).  The limit is
+// counted in polls and in SM cycles (clock64 is a register read).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
+  long long t0 = 0;
   for (uint32_t polls = 1; polls < kWaitLimitPolls; ++polls) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((polls & 0xff) == 0) {
+    if ((polls & 0x3f) == 0) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) break;
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitCycles) break;
     }
   }
   *abort_flag = 1;

@@ -63,7 +63,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int64_t m0 = (int64_t)blockIdx.x * BM, n0 = (int64_t)blockIdx.y * BN;
+  // blockIdx.x walks the N tiles first: the CTAs of one wave share a few A row blocks (the large,
+  // token-sized operand is then read from HBM once) and sweep all of B (weights, L2 resident).
+  const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
   const int num_kb = (int)((p.K + BK - 1) / BK);
 
   if (threadIdx.x == 0) {
@@ -115,23 +117,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc_bf16(BM, BN, AMODE == A_MN, BMODE == B_MN);
+      // Descriptors are built once; a stage or K step only adds to the 14-bit start-address
+      // field (16-byte units), which never carries out of it.
+      const uint64_t adesc0 = (AMODE == A_MN) ? smem_desc_sw128(sbase, SLAB_BYTES, 1024) : smem_desc_sw128(sbase, 16, 1024);
+      const uint64_t bdesc0 = (BMODE == B_MN) ? smem_desc_sw128(sbase + A_BYTES, SLAB_BYTES, 1024)
+                                              : smem_desc_sw128(sbase + A_BYTES, 16, 1024);
+      constexpr uint32_t a_kstep = ((AMODE == A_MN) ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+      constexpr uint32_t b_kstep = ((BMODE == B_MN) ? UMMA_K * 128 : UMMA_K * 2) >> 4;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
+      int s = 0;
+      uint32_t ph = 0;
+      for (int kb = 0; kb < num_kb; ++kb) {
         ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a_smem = sbase + s * STAGE_BYTES, b_smem = a_smem + A_BYTES;
+        const uint64_t ad = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
+        const uint64_t bd = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
 #pragma unroll
-        for (int j = 0; j < BK / UMMA_K; ++j) {
-          const uint64_t adesc = (AMODE == A_MN) ? smem_desc_sw128(a_smem + j * (UMMA_K * 128), SLAB_BYTES, 1024)
-                                                 : smem_desc_sw128(a_smem + j * (UMMA_K * 2), 16, 1024);
-          const uint64_t bdesc = (BMODE == B_MN) ? smem_desc_sw128(b_smem + j * (UMMA_K * 128), SLAB_BYTES, 1024)
-                                                 : smem_desc_sw128(b_smem + j * (UMMA_K * 2), 16, 1024);
-          umma_bf16(tmem_base, adesc, bdesc, idesc, (kb | j) != 0 ? 1u : 0u);
-        }
+        for (int j = 0; j < BK / UMMA_K; ++j)
+          umma_bf16(tmem_base, ad + j * a_kstep, bd + j * b_kstep, idesc, (kb | j) != 0 ? 1u : 0u);
         umma_commit(empty_bar(s));
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
       }
       if (ok) umma_commit(accfull_bar);
     }
@@ -183,8 +189,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   // ---------------------------------------------------------------- teardown
   if (*abort_flag) {
     // give copies that may still be in flight time to land before the CTA's shared memory is released
-    const unsigned long long t0 = global_ns();
-    while (global_ns() - t0 < 1000000ull) __nanosleep(1000);
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) __nanosleep(1000);
   }
   tc_fence_before();
   __syncthreads();

@@ -40,17 +40,113 @@ constexpr int SK_TILE_ELEMS = SK_BM * SK_BN;         // fp32 elements of one par
 constexpr int SK_MAX_CTAS = 148;                     // grid size used for workspace sizing
 
 // Static schedule shared by the sketch kernel, the reduce kernel and the host.
+//
+// Units are (tile, 64-token step) pairs; every CTA gets `upc` consecutive units of a
+// line that is ordered so that CTAs running at the same time read the same token rows
+// of B (they then come out of L2 instead of being fetched from HBM once per tile row):
+//   1. rounds: while at least num_ctas tiles are left, CTA i takes one whole tile;
+//   2. the remaining `tiles_rem` tiles are cut along tokens into blocks of `upc` steps;
+//      block b of tile t goes to CTA b * tiles_rem + t, so all CTAs of a block walk the
+//      same token range in step;
+//   3. the last, narrower block (width `w_last`) is laid out tile after tile and cut
+//      into ranges of `upc` units, which may span several tiles.
+// Every (CTA, tile) intersection is one segment = one fp32 partial tile (slot).
 struct SketchSchedule {
-  int tiles_m, tiles_n, ksteps;       // output tiles and 64-token steps per tile
-  int num_ctas;
-  long long total_units, units_per_cta, lcm_units;   // lcm(units_per_cta, ksteps)
-  __host__ __device__ long long slot_of(int cta, int tile, long long seg_start) const {
-    // Segments are numbered in unit order; one starts at every CTA-range start and at
-    // every tile start (a unit that is both counts once).
-    return (long long)cta + tile - seg_start / lcm_units;
+  int tiles_m, tiles_n, ksteps;
+  int num_ctas;            // grid size
+  int rounds;              // whole-tile rounds
+  int tiles_rem;           // tiles handled by the blocked part
+  int upc;                 // units per CTA in the blocked part
+  int full_blocks;         // blocks of width upc
+  int w_last;              // width of the last block (0 if none)
+  long long lcm_last;      // lcm(upc, w_last)
+
+  __host__ __device__ int tiles() const { return tiles_m * tiles_n; }
+  __host__ __device__ long long num_slots() const { return (long long)tiles() + num_ctas; }
+  // slot of the whole-tile segment of a round
+  __host__ __device__ long long slot_round(int tile) const { return tile; }
+  // slot of full block b of remainder tile t (CTA b * tiles_rem + t)
+  __host__ __device__ long long slot_block(int b, int t) const {
+    return (long long)rounds * num_ctas + (long long)b * tiles_rem + t;
   }
-  __host__ __device__ long long num_slots() const { return (long long)num_ctas + (long long)tiles_m * tiles_n; }
+  // slot of a segment of the last block: CTA index ci and tile t, both relative to the last
+  // block, seg_start = first unit of the segment in the last block's tile-major line.
+  // Segments are numbered in line order; one starts at every CTA-range start and at every
+  // tile start (a unit that is both counts once).
+  __host__ __device__ long long slot_last(int ci, int t, long long seg_start) const {
+    return (long long)rounds * num_ctas + (long long)full_blocks * tiles_rem + ci + t - seg_start / lcm_last;
+  }
 };
+
+// One segment of work of a CTA.
+struct SketchSegment {
+  int tile, ks0, ks1;
+  long long slot;
+};
+
+// Enumerates the segments of CTA `cta` in execution order; returns false when exhausted.
+// `it` and `cursor` are the iteration state (start both at 0).
+__host__ __device__ inline bool sketch_next_segment(const SketchSchedule& sc, int cta, int& it, long long& cursor,
+                                                    SketchSegment& seg) {
+  if (it < sc.rounds) {                       // whole tiles
+    seg.tile = it * sc.num_ctas + cta;
+    seg.ks0 = 0; seg.ks1 = sc.ksteps;
+    seg.slot = sc.slot_round(seg.tile);
+    ++it;
+    return true;
+  }
+  if (sc.tiles_rem == 0) return false;
+  const int base_tile = sc.rounds * sc.num_ctas;
+  const int nfull = sc.full_blocks * sc.tiles_rem;       // CTAs that own a full block
+  if (cta < nfull) {
+    if (it > sc.rounds) return false;
+    const int b = cta / sc.tiles_rem, t = cta % sc.tiles_rem;
+    seg.tile = base_tile + t;
+    seg.ks0 = b * sc.upc; seg.ks1 = seg.ks0 + sc.upc;
+    seg.slot = sc.slot_block(b, t);
+    ++it;
+    return true;
+  }
+  if (sc.w_last == 0) return false;
+  const int ci = cta - nfull;
+  const long long total = (long long)sc.tiles_rem * sc.w_last;
+  const long long begin = (long long)ci * sc.upc;
+  const long long end = begin + sc.upc < total ? begin + sc.upc : total;
+  if (it == sc.rounds) { cursor = begin; }
+  if (cursor >= end) return false;
+  const int t = (int)(cursor / sc.w_last);
+  const int off = (int)(cursor % sc.w_last);
+  const long long rem = end - cursor;
+  const int len = (int)((sc.w_last - off < rem) ? sc.w_last - off : rem);
+  seg.tile = base_tile + t;
+  seg.ks0 = sc.full_blocks * sc.upc + off;
+  seg.ks1 = seg.ks0 + len;
+  seg.slot = sc.slot_last(ci, t, cursor);
+  cursor += len;
+  ++it;
+  return true;
+}
+
+// Calls f(slot) for every partial tile of output tile `tile`, in schedule order (the order in
+// which sketch_reduce_kernel adds them).
+template <class F>
+__host__ __device__ inline void sketch_for_each_slot_of_tile(const SketchSchedule& sc, int tile, F&& f) {
+  const int base_tile = sc.rounds * sc.num_ctas;
+  if (tile < base_tile) {
+    f(sc.slot_round(tile));
+    return;
+  }
+  const int t = tile - base_tile;
+  for (int b = 0; b < sc.full_blocks; ++b) f(sc.slot_block(b, t));
+  if (sc.w_last > 0) {
+    const int ci_first = (int)(((long long)t * sc.w_last) / sc.upc);
+    const int ci_last = (int)((((long long)t + 1) * sc.w_last - 1) / sc.upc);
+    for (int ci = ci_first; ci <= ci_last; ++ci) {
+      const long long cs = (long long)ci * sc.upc, ts = (long long)t * sc.w_last;
+      f(sc.slot_last(ci, t, cs > ts ? cs : ts));
+    }
+  }
+}
 
 inline long long gcd_ll(long long a, long long b) { while (b) { long long t = a % b; a = b; b = t; } return a; }
 
@@ -59,11 +155,22 @@ inline SketchSchedule make_sketch_schedule(long long rows, long long cols, long 
   s.tiles_m = (int)((rows + SK_BM - 1) / SK_BM);
   s.tiles_n = (int)((cols + SK_BN - 1) / SK_BN);
   s.ksteps = (int)((tokens + SK_AK - 1) / SK_AK);
-  s.total_units = (long long)s.tiles_m * s.tiles_n * s.ksteps;
-  s.num_ctas = (int)(s.total_units < max_ctas ? s.total_units : max_ctas);
-  s.units_per_cta = (s.total_units + s.num_ctas - 1) / s.num_ctas;
-  s.num_ctas = (int)((s.total_units + s.units_per_cta - 1) / s.units_per_cta);
-  s.lcm_units = s.units_per_cta / gcd_ll(s.units_per_cta, s.ksteps) * s.ksteps;
+  const int tiles = s.tiles_m * s.tiles_n;
+  s.rounds = tiles / max_ctas;
+  s.tiles_rem = tiles % max_ctas;
+  s.num_ctas = max_ctas;
+  s.upc = 0; s.full_blocks = 0; s.w_last = 0; s.lcm_last = 1;
+  if (s.tiles_rem > 0) {
+    const long long total = (long long)s.tiles_rem * s.ksteps;
+    s.upc = (int)((total + max_ctas - 1) / max_ctas);
+    if (s.upc < 4 && s.upc < s.ksteps) s.upc = s.ksteps < 4 ? s.ksteps : 4;   // no slivers
+    s.full_blocks = s.ksteps / s.upc;
+    s.w_last = s.ksteps - s.full_blocks * s.upc;
+    if (s.w_last > 0) s.lcm_last = (long long)s.upc / gcd_ll(s.upc, s.w_last) * s.w_last;
+    const long long last_ctas = s.w_last > 0 ? ((long long)s.tiles_rem * s.w_last + s.upc - 1) / s.upc : 0;
+    const long long used = (long long)s.full_blocks * s.tiles_rem + last_ctas;
+    if (s.rounds == 0) s.num_ctas = (int)used;          // never more than max_ctas by construction of upc
+  }
   return s;
 }
 
@@ -145,12 +252,11 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const SketchSchedule& sc = p.sched;
-  const long long u_begin = (long long)blockIdx.x * sc.units_per_cta;
-  const long long u_end = (u_begin + sc.units_per_cta < sc.total_units) ? u_begin + sc.units_per_cta : sc.total_units;
+  const int cta = (int)blockIdx.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < SK_A_STAGES; ++s) {
-      mbar_init(fulla_bar(s), SK_GEN_THREADS);
+      mbar_init(fulla_bar(s), SK_GEN_WARPS);      // one arrival per generator warp
       mbar_init(emptya_bar(s), 1);
     }
     for (int s = 0; s < SK_B_STAGES; ++s) {
@@ -158,7 +264,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       mbar_init(emptyb_bar(s), 1);
     }
     mbar_init(accfull_bar, 1);
-    mbar_init(accempty_bar, SK_GEN_THREADS);
+    mbar_init(accempty_bar, SK_GEN_WARPS);
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -175,28 +281,27 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     // ------------------------------------------------------------ TMA producer (B)
     if (lane == 0) {
       tma_prefetch_desc(&tmB);
-      long long it = 0;   // running 32-token stage counter
+      int s = 0;
+      uint32_t ph = 0;
       bool ok = true;
-      for (long long u = u_begin; u < u_end && ok;) {
-        const int tile = (int)(u / sc.ksteps);
-        const int ks0 = (int)(u % sc.ksteps);
-        const long long rem = u_end - u;
-        const int ks1 = (int)((sc.ksteps - ks0 < rem) ? sc.ksteps : ks0 + rem);
-        const int n0 = (tile % sc.tiles_n) * SK_BN;
-        for (int ks = ks0; ks < ks1 && ok; ++ks) {
-          for (int half = 0; half < 2; ++half, ++it) {
-            const int s = (int)(it % SK_B_STAGES);
-            const uint32_t ph = (uint32_t)(it / SK_B_STAGES) & 1u;
+      int seg_it = 0;
+      long long cursor = 0;
+      SketchSegment sg;
+      while (ok && sketch_next_segment(sc, cta, seg_it, cursor, sg)) {
+        const int n0 = (sg.tile % sc.tiles_n) * SK_BN;
+        for (int ks = sg.ks0; ks < sg.ks1 && ok; ++ks) {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
             if (!mbar_wait(emptyb_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-            const uint32_t b_smem = smem_u32(b_ring + s * SK_B_BYTES);
+            const uint32_t b_smem = smem_u32(b_ring) + s * SK_B_BYTES;
             mbar_arrive_expect_tx(fullb_bar(s), SK_B_BYTES);
             const int tok0 = ks * SK_AK + half * SK_BK;
 #pragma unroll
             for (int sl = 0; sl < SK_BN / 64; ++sl)
               tma_load_2d(b_smem + sl * SK_B_SLAB, &tmB, fullb_bar(s), n0 + 64 * sl, tok0);
+            if (++s == SK_B_STAGES) { s = 0; ph ^= 1u; }
           }
         }
-        u += ks1 - ks0;
       }
     }
     __syncwarp();
@@ -204,44 +309,49 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc_bf16(SK_BM, 256, false, true);
-      long long ita = 0, itb = 0;
+      // One thread issues everything: descriptors are built once, stage and K-step offsets are
+      // added to the start-address field (16-byte units).
+      const uint64_t adesc0 = smem_desc_sw128(smem_u32(a_ring), 16, 1024);
+      const uint64_t bdesc0 = smem_desc_sw128(smem_u32(b_ring), SK_B_SLAB, 1024);
+      int sa = 0, sb = 0;
+      uint32_t pha = 0, phb = 0;
       int seg = 0;
       bool ok = true;
-      for (long long u = u_begin; u < u_end && ok; ++seg) {
-        const int ks0 = (int)(u % sc.ksteps);
-        const long long rem = u_end - u;
-        const int ks1 = (int)((sc.ksteps - ks0 < rem) ? sc.ksteps : ks0 + rem);
+      int seg_it = 0;
+      long long cursor = 0;
+      SketchSegment sg;
+      for (; ok && sketch_next_segment(sc, cta, seg_it, cursor, sg); ++seg) {
         if (seg > 0) {   // the previous segment's accumulator must have been drained
           ok = mbar_wait(accempty_bar, (uint32_t)(seg - 1) & 1u, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
         }
-        for (int ks = ks0; ks < ks1 && ok; ++ks, ++ita) {
-          const int sa = (int)(ita % SK_A_STAGES);
-          ok = mbar_wait(fulla_bar(sa), (uint32_t)(ita / SK_A_STAGES) & 1u, abort_flag, p.status);
+        uint32_t acc = 0;
+        for (int ks = sg.ks0; ks < sg.ks1 && ok; ++ks) {
+          ok = mbar_wait(fulla_bar(sa), pha, abort_flag, p.status);
           if (!ok) break;
-          const uint32_t a_smem = smem_u32(a_ring + sa * SK_A_BYTES);
-          for (int half = 0; half < 2; ++half, ++itb) {
-            const int sb = (int)(itb % SK_B_STAGES);
-            ok = mbar_wait(fullb_bar(sb), (uint32_t)(itb / SK_B_STAGES) & 1u, abort_flag, p.status);
+          const uint64_t ad = adesc0 + (uint64_t)(sa * (SK_A_BYTES >> 4));
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            ok = mbar_wait(fullb_bar(sb), phb, abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t b_smem = smem_u32(b_ring + sb * SK_B_BYTES);
+            const uint64_t bd = bdesc0 + (uint64_t)(sb * (SK_B_BYTES >> 4));
 #pragma unroll
             for (int j = 0; j < SK_BK / 16; ++j) {
-              const uint64_t adesc = smem_desc_sw128(a_smem + (half * (SK_BK / 16) + j) * 32, 16, 1024);
 #pragma unroll
-              for (int nh = 0; nh < 2; ++nh) {
-                const uint64_t bdesc = smem_desc_sw128(b_smem + nh * 4 * SK_B_SLAB + j * 2048, SK_B_SLAB, 1024);
-                umma_bf16(tmem_base + nh * 256, adesc, bdesc, idesc, (ks > ks0 || half > 0 || j > 0) ? 1u : 0u);
-              }
+              for (int nh = 0; nh < 2; ++nh)
+                umma_bf16(tmem_base + nh * 256, ad + (half * (SK_BK / 16) + j) * 2,
+                          bd + ((nh * 4 * SK_B_SLAB + j * 2048) >> 4), idesc, acc);
+              acc = 1;
             }
             umma_commit(emptyb_bar(sb));
+            if (++sb == SK_B_STAGES) { sb = 0; phb ^= 1u; }
           }
           if (ok) umma_commit(emptya_bar(sa));
+          if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
         }
         if (ok) umma_commit(accfull_bar);
-        u += ks1 - ks0;
       }
     }
     __syncwarp();
@@ -249,21 +359,23 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     // ------------------------------------------------------------ S generators + accumulator drain
     const int gtid = threadIdx.x - 64;
     const int gw = warp - 2;
-    long long ita = 0;
+    int sa = 0;
+    uint32_t pha = 0;
     int seg = 0;
     bool ok = true;
-    for (long long u = u_begin; u < u_end && ok; ++seg) {
-      const int tile = (int)(u / sc.ksteps);
-      const int ks0 = (int)(u % sc.ksteps);
-      const long long rem = u_end - u;
-      const int ks1 = (int)((sc.ksteps - ks0 < rem) ? sc.ksteps : ks0 + rem);
+    int seg_it = 0;
+    long long cursor = 0;
+    SketchSegment sg;
+    for (; ok && sketch_next_segment(sc, cta, seg_it, cursor, sg); ++seg) {
+      const int tile = sg.tile;
       const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
-      for (int ks = ks0; ks < ks1; ++ks, ++ita) {
-        const int sa = (int)(ita % SK_A_STAGES);
-        if (!mbar_wait(emptya_bar(sa), ((uint32_t)(ita / SK_A_STAGES) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+      for (int ks = sg.ks0; ks < sg.ks1; ++ks) {
+        if (!mbar_wait(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)) { ok = false; break; }
         sketch_generate_stage(a_ring + sa * SK_A_BYTES, pk, p, m0, (long long)ks * SK_AK, gtid);
         fence_proxy_async_smem();
-        mbar_arrive(fulla_bar(sa));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(fulla_bar(sa));
+        if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
       }
       ok = __all_sync(0xffffffffu, ok && mbar_wait(accfull_bar, (uint32_t)seg & 1u, abort_flag, p.status));
       if (!ok) break;
@@ -271,8 +383,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       {
         const int q = warp & 3;                 // tensor-memory lane quarter of this warp
         const int cgroup = gw >> 2;             // 4 warps share a quarter: 128 columns each
-        const long long seg_start = u;
-        float* slot = p.partial + sc.slot_of((int)blockIdx.x, tile, seg_start) * (long long)SK_TILE_ELEMS;
+        float* slot = p.partial + sg.slot * (long long)SK_TILE_ELEMS;
         float* prow = slot + (long long)(q * 32 + lane) * SK_BN;
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
@@ -286,14 +397,15 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
         }
       }
       tc_fence_before();
-      mbar_arrive(accempty_bar);
-      u += ks1 - ks0;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(accempty_bar);
     }
   }
   // ---------------------------------------------------------------- teardown
   if (*abort_flag) {
-    const unsigned long long t0 = global_ns();
-    while (global_ns() - t0 < 1000000ull) __nanosleep(1000);
+    // give copies that may still be in flight time to land before the shared memory is released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) __nanosleep(1000);
   }
   tc_fence_before();
   __syncthreads();
@@ -308,8 +420,6 @@ sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ ou
   const SketchSchedule& sc = p.sched;
   const int tile = blockIdx.x;
   const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM, n0 = (long long)(tile % sc.tiles_n) * SK_BN;
-  const long long t_begin = (long long)tile * sc.ksteps, t_end = t_begin + sc.ksteps;
-  const int c_first = (int)(t_begin / sc.units_per_cta), c_last = (int)((t_end - 1) / sc.units_per_cta);
   const int col = threadIdx.x * 4;
   if (n0 + col >= p.cols) return;
   for (int rr = 0; rr < SKR_ROWS; ++rr) {
@@ -317,13 +427,11 @@ sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ ou
     const long long j = m0 + r;
     if (j >= p.rows) break;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = c_first; c <= c_last; ++c) {
-      const long long cs = (long long)c * sc.units_per_cta;
-      const long long seg_start = cs > t_begin ? cs : t_begin;
-      const float* slot = p.partial + sc.slot_of(c, tile, seg_start) * (long long)SK_TILE_ELEMS;
+    sketch_for_each_slot_of_tile(sc, tile, [&](long long slot_index) {
+      const float* slot = p.partial + slot_index * (long long)SK_TILE_ELEMS;
       const float4 v = *reinterpret_cast<const float4*>(slot + (long long)r * SK_BN + col);
       acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-    }
+    });
     const bool is_ones = p.ones_row && j == p.b_proj;
     const float s = is_ones ? 1.0f : scale;
     __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * s, acc.y * s), hi = __floats2bfloat162_rn(acc.z * s, acc.w * s);

@@ -80,6 +80,8 @@ WORKLOADS = {w.name: w for w in [
     # RoBERTa-large
     _w("large_ffn_up_rho0.1", DTYPE_BF16, 16384, 1024, 4096, 0.1, DIST_GAUSSIAN, 7),
     _w("large_ffn_down_rho0.1", DTYPE_BF16, 16384, 4096, 1024, 0.1, DIST_GAUSSIAN, 8),
+    # diagnostic: the RoBERTa-large shape with the cheap sketch distribution (isolates the cost of the normals)
+    _w("large_ffn_up_rad_rho0.1", DTYPE_BF16, 16384, 1024, 4096, 0.1, DIST_RADEMACHER, 9),
 ]}
 
 

@@ -93,4 +93,45 @@ def test_no_device_is_an_error_not_a_fallback(lib):
     fwd = lib.rmm_forward
     fwd.argtypes = [vp, vp, vp, i64, i64, i64, C.c_uint64, i64, C.c_int, C.c_int, vp, vp, vp, C.c_size_t, vp]
     p = 4096
-    assert fwd(p, p, None, 8, 8, 8, 0, 4, 0, 0, p, p, p, 1 << 20, None) == 4
+    assert fwd(p, p, None, 8, 8, 8, 0, 4, 0, 0, p, p, p, 1 << 40, None) == 4
+
+
+@pytest.mark.parametrize("rows,cols,tokens,ctas", [
+    (1639, 4096, 16384, 148), (1638, 1024, 16384, 148), (820, 3072, 4096, 148), (819, 768, 4096, 148),
+    (3687, 3072, 4096, 148), (5, 24, 37, 148), (131, 520, 300, 148), (1, 8, 1, 148), (2049, 768, 4096, 148),
+    (1153, 4096, 4096, 74), (1639, 4096, 16384, 7), (300, 1500, 1000, 3), (129, 513, 65, 74),
+    (7000, 3072, 4096, 74), (40000, 3072, 4096, 148),
+])
+def test_sketch_schedule_covers_every_unit_once(rows, cols, tokens, ctas):
+    """Host logic of the sketch kernels' stream-K schedule: every (tile, token step) unit belongs to
+    exactly one segment, no two segments share a partial-tile slot, and the reduction's slot list
+    per tile is exactly the set of slots that the kernel writes for that tile."""
+    import collections
+
+    import paper_2201_13195_b200 as P
+    segs, info = P.rmm_debug_sketch_schedule(rows, cols, tokens, ctas, mode=0)
+    red, info2 = P.rmm_debug_sketch_schedule(rows, cols, tokens, ctas, mode=1)
+    assert info == info2
+    tiles, ksteps = info["tiles"], info["ksteps"]
+    assert tiles == -(-rows // 128) * -(-cols // 512) and ksteps == -(-tokens // 64)
+    assert info["num_ctas"] <= ctas
+    cover = collections.Counter()
+    slots = set()
+    by_tile = collections.defaultdict(list)
+    per_cta = collections.Counter()
+    for cta, tile, ks0, ks1, slot in segs:
+        assert 0 <= cta < info["num_ctas"] and 0 <= tile < tiles and 0 <= ks0 < ks1 <= ksteps
+        assert 0 <= slot < info["num_slots"] and slot not in slots
+        slots.add(slot)
+        by_tile[tile].append(slot)
+        per_cta[cta] += ks1 - ks0
+        for ks in range(ks0, ks1):
+            cover[(tile, ks)] += 1
+    assert len(cover) == tiles * ksteps and set(cover.values()) == {1}
+    red_by_tile = collections.defaultdict(list)
+    for tile, slot, *_ in red:
+        red_by_tile[tile].append(slot)
+    assert {t: sorted(v) for t, v in by_tile.items()} == {t: sorted(v) for t, v in red_by_tile.items()}
+    # balance: no CTA carries much more than the mean
+    mean = tiles * ksteps / info["num_ctas"]
+    assert max(per_cta.values()) <= mean + (ksteps if tiles >= ctas else 4) + 1

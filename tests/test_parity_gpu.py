@@ -29,6 +29,18 @@ def test_sketch_dump_bit_exact(dtype, dist, N, k, seed):
     assert np.array_equal(got.to(torch.float32).cpu().numpy(), want)
 
 
+def test_gaussian_transform_bit_exact_on_all_radius_and_angle_inputs():
+    """Every one of the 2^16 radius inputs (with three angle patterns) and of the 2^16 angle
+    inputs (with three radius patterns) of the uniform -> normal map, bit for bit."""
+    P = _P()
+    hi = np.arange(65536, dtype=np.uint64)
+    words = np.concatenate([(hi << 16) | lo for lo in (16383, 0x8001, 0x5A5A)] +
+                           [(np.uint64(h) << 16) | hi for h in (0, 20000, 65535)]).astype(np.uint32)
+    got = P.rmm_debug_gauss_words(torch.from_numpy(words.view(np.int32)).cuda()).cpu().numpy()
+    want = np.array([O.gauss_pair(int(w)) for w in words], dtype=np.float32)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
 @pytest.mark.parametrize("dtype", [R.DTYPE_BF16, R.DTYPE_F32])
 @pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER])
 def test_production_kernel_sketch_bit_exact(dtype, dist):
