@@ -150,7 +150,9 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   tc::GemmParams p;
   p.M = M; p.N = N; p.K = K;
   p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.status = status;
-  dim3 grid((unsigned)((N + tc::BN - 1) / tc::BN), (unsigned)((M + tc::BM - 1) / tc::BM));
+  const int64_t tiles = ((N + tc::BN - 1) / tc::BN) * ((M + tc::BM - 1) / tc::BM);
+  const int sms = device_state().num_sms;
+  dim3 grid((unsigned)(tiles < sms ? tiles : sms));   // persistent: one CTA per SM
   tc::gemm_kernel<AMODE, BMODE><<<grid, 64 + 32 * tc::NEPI, tc::GEMM_SMEM_BYTES, stream>>>(tmA, tmB, p);
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
@@ -173,7 +175,7 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   const int sms = device_state().num_sms;
   p.sched = tc::make_sketch_schedule(p.rows, cols, tokens, sms < tc::SK_MAX_CTAS ? sms : tc::SK_MAX_CTAS);
   tc::sketch_kernel<<<p.sched.num_ctas, tc::SK_THREADS, tc::SK_SMEM_BYTES, stream>>>(tmB, p, pk);
-  dim3 rgrid((unsigned)p.sched.tiles(), tc::SK_BM / tc::SKR_ROWS);
+  dim3 rgrid((unsigned)p.sched.tiles(), tc::SK_BM);
   tc::sketch_reduce_kernel<<<rgrid, 128, 0, stream>>>(p, c, reinterpret_cast<__nv_bfloat16*>(out),
                                                       reinterpret_cast<__nv_bfloat16*>(ones_out));
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;

@@ -1,5 +1,5 @@
 // Tensor-core contraction kernel for the bf16 mode (sm_100a): C = alpha * A B^T (+ bias),
-// bf16 operands, fp32 accumulation in tensor memory, one 128 x 256 output tile per CTA.
+// bf16 operands, fp32 accumulation in tensor memory, 128 x 256 output tiles, persistent CTAs.
 //
 // The three dense contractions of Algorithm 1 whose operands all live in memory differ only
 // in the operand layouts (the two sketch contractions are in tc_sketch.cuh):
@@ -13,7 +13,8 @@
 // Warp roles: warp 0 = TMA producer, warp 1 = tensor-memory owner and MMA issuer,
 // warps 2..5 = epilogue.  Stages of a ring of shared-memory buffers are handed over with
 // mbarriers: full (TMA bytes landed), empty (tcgen05.commit: the MMAs that read the stage
-// have retired), accfull (all MMAs of the tile retired).
+// have retired), accfull (all MMAs of the tile retired), accempty (the epilogue has read the
+// accumulator buffer out of tensor memory).
 #pragma once
 #include "tc_common.cuh"
 
@@ -26,7 +27,7 @@ constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;          // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SLAB_BYTES = 64 * BK * 2;       // one [64 k][64 mn] MN-major slab, 8 KiB
-constexpr int TMEM_COLS = 256;
+constexpr int TMEM_COLS = 512;              // two 128 x 256 fp32 accumulators: MMAs of tile i+1 overlap the epilogue of tile i
 constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 enum : int { A_K = 0, A_MN = 1 };
@@ -58,14 +59,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
-  const uint32_t accfull_bar = bar0 + 8u * (2 * STAGES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
+  auto accfull_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
+  auto accempty_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // blockIdx.x walks the N tiles first: the CTAs of one wave share a few A row blocks (the large,
+  // Persistent: this CTA takes tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Tile t is
+  // (m = t / tiles_n, n = t % tiles_n): the CTAs of one wave share a few A row blocks (the large,
   // token-sized operand is then read from HBM once) and sweep all of B (weights, L2 resident).
-  const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
+  const int tiles_n = (int)((p.N + BN - 1) / BN);
+  const int num_tiles = (int)((p.M + BM - 1) / BM) * tiles_n;
   const int num_kb = (int)((p.K + BK - 1) / BK);
 
   if (threadIdx.x == 0) {
@@ -73,7 +77,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
-    mbar_init(accfull_bar, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(accfull_bar(b), 1);
+      mbar_init(accempty_bar(b), NEPI);     // one arrival per epilogue warp
+    }
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -91,24 +98,29 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (lane == 0) {
       tma_prefetch_desc(&tmA);
       tma_prefetch_desc(&tmB);
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) break;
-        const uint32_t a_smem = sbase + s * STAGE_BYTES, b_smem = a_smem + A_BYTES;
-        mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES);
-        const int k0 = kb * BK;
-        if (AMODE == A_K) {
-          tma_load_2d(a_smem, &tmA, full_bar(s), k0, (int)m0);
-        } else {
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t a_smem = sbase + s * STAGE_BYTES, b_smem = a_smem + A_BYTES;
+          mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES);
+          const int k0 = kb * BK;
+          if (AMODE == A_K) {
+            tma_load_2d(a_smem, &tmA, full_bar(s), k0, m0);
+          } else {
 #pragma unroll
-          for (int sl = 0; sl < BM / 64; ++sl) tma_load_2d(a_smem + sl * SLAB_BYTES, &tmA, full_bar(s), (int)m0 + 64 * sl, k0);
-        }
-        if (BMODE == B_K) {
-          tma_load_2d(b_smem, &tmB, full_bar(s), k0, (int)n0);
-        } else {
+            for (int sl = 0; sl < BM / 64; ++sl) tma_load_2d(a_smem + sl * SLAB_BYTES, &tmA, full_bar(s), m0 + 64 * sl, k0);
+          }
+          if (BMODE == B_K) {
+            tma_load_2d(b_smem, &tmB, full_bar(s), k0, n0);
+          } else {
 #pragma unroll
-          for (int sl = 0; sl < BN / 64; ++sl) tma_load_2d(b_smem + sl * SLAB_BYTES, &tmB, full_bar(s), (int)n0 + 64 * sl, k0);
+            for (int sl = 0; sl < BN / 64; ++sl) tma_load_2d(b_smem + sl * SLAB_BYTES, &tmB, full_bar(s), n0 + 64 * sl, k0);
+          }
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
       }
     }
@@ -127,35 +139,48 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       bool ok = true;
       int s = 0;
       uint32_t ph = 0;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
+      int it = 0;                               // tiles done by this CTA
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+        const int buf = it & 1;
+        // the epilogue must have drained this accumulator buffer (two tiles ago)
+        ok = mbar_wait(accempty_bar(buf), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
-        const uint64_t ad = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
-        const uint64_t bd = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t ad = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
+          const uint64_t bd = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
 #pragma unroll
-        for (int j = 0; j < BK / UMMA_K; ++j)
-          umma_bf16(tmem_base, ad + j * a_kstep, bd + j * b_kstep, idesc, (kb | j) != 0 ? 1u : 0u);
-        umma_commit(empty_bar(s));
-        if (++s == STAGES) { s = 0; ph ^= 1u; }
+          for (int j = 0; j < BK / UMMA_K; ++j)
+            umma_bf16(d_tmem, ad + j * a_kstep, bd + j * b_kstep, idesc, (kb | j) != 0 ? 1u : 0u);
+          umma_commit(empty_bar(s));
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (ok) umma_commit(accfull_bar(buf));
       }
-      if (ok) umma_commit(accfull_bar);
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ epilogue
-    const bool acc_ready = __all_sync(0xffffffffu, mbar_wait(accfull_bar, 0u, abort_flag, p.status));
-    if (acc_ready) {
+    // ------------------------------------------------------------ epilogue (overlaps the next tile's MMAs)
+    const int q = warp & 3;                       // tensor-memory lane quarter this warp may read
+    const __nv_bfloat16* bias = reinterpret_cast<const __nv_bfloat16*>(p.bias);
+    int it = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+      const int buf = it & 1;
+      const bool acc_ready =
+          __all_sync(0xffffffffu, mbar_wait(accfull_bar(buf), (uint32_t)(it >> 1) & 1u, abort_flag, p.status));
+      if (!acc_ready) break;
       tc_fence_after();
-      const int q = warp & 3;                       // tensor-memory lane quarter this warp may read
-      constexpr int CHUNKS = BN / 32;
+      const int64_t m0 = (int64_t)(tile / tiles_n) * BM, n0 = (int64_t)(tile % tiles_n) * BN;
       const int64_t row = m0 + q * 32 + lane;
       __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc;
-      const __nv_bfloat16* bias = reinterpret_cast<const __nv_bfloat16*>(p.bias);
-      for (int cc = 0; cc < CHUNKS; ++cc) {
-        const int c = cc;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
         uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
+        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), v);
         tmem_ld_wait();
         if (row < p.M) {
 #pragma unroll
@@ -184,6 +209,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
         }
       }
+      // hand the buffer back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(accempty_bar(buf));
     }
   }
   // ---------------------------------------------------------------- teardown

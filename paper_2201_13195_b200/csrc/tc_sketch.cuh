@@ -413,35 +413,46 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
 }
 
 // Adds the partial tiles of each output tile in schedule order, scales, rounds to bf16.
-// grid = (tiles, 128 / SKR_ROWS), block = 128 threads: thread t owns columns 4t .. 4t+3.
-constexpr int SKR_ROWS = 8;
+// grid = (tiles, 128 rows), block = 128 threads: thread t owns columns 4t .. 4t+3 of one row.
+// All loads of a thread are independent, so the kernel runs at memory speed.
+constexpr int SKR_MAX_SLOTS = 8;     // partial tiles summed per batch of loads
 __global__ void __launch_bounds__(128)
 sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ ones_out) {
   const SketchSchedule& sc = p.sched;
   const int tile = blockIdx.x;
   const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM, n0 = (long long)(tile % sc.tiles_n) * SK_BN;
+  const int r = blockIdx.y;
+  const long long j = m0 + r;
   const int col = threadIdx.x * 4;
-  if (n0 + col >= p.cols) return;
-  for (int rr = 0; rr < SKR_ROWS; ++rr) {
-    const int r = blockIdx.y * SKR_ROWS + rr;
-    const long long j = m0 + r;
-    if (j >= p.rows) break;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    sketch_for_each_slot_of_tile(sc, tile, [&](long long slot_index) {
-      const float* slot = p.partial + slot_index * (long long)SK_TILE_ELEMS;
-      const float4 v = *reinterpret_cast<const float4*>(slot + (long long)r * SK_BN + col);
-      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-    });
-    const bool is_ones = p.ones_row && j == p.b_proj;
-    const float s = is_ones ? 1.0f : scale;
-    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * s, acc.y * s), hi = __floats2bfloat162_rn(acc.z * s, acc.w * s);
-    uint2 o = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-    // cols is a multiple of 8 and col a multiple of 4: the 4 columns are all inside or all outside
-    if (is_ones) {
-      if (ones_out) *reinterpret_cast<uint2*>(ones_out + n0 + col) = o;
-    } else {
-      *reinterpret_cast<uint2*>(out + j * p.cols + n0 + col) = o;
-    }
+  if (j >= p.rows || n0 + col >= p.cols) return;
+  long long slots[SKR_MAX_SLOTS];
+  int ns = 0;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  const long long off = (long long)r * SK_BN + col;
+  auto flush = [&]() {
+    float4 v[SKR_MAX_SLOTS];
+#pragma unroll
+    for (int i = 0; i < SKR_MAX_SLOTS; ++i)
+      if (i < ns) v[i] = __ldcs(reinterpret_cast<const float4*>(p.partial + slots[i] * (long long)SK_TILE_ELEMS + off));
+#pragma unroll
+    for (int i = 0; i < SKR_MAX_SLOTS; ++i)
+      if (i < ns) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
+    ns = 0;
+  };
+  sketch_for_each_slot_of_tile(sc, tile, [&](long long slot_index) {
+    slots[ns++] = slot_index;
+    if (ns == SKR_MAX_SLOTS) flush();
+  });
+  flush();
+  const bool is_ones = p.ones_row && j == p.b_proj;
+  const float s = is_ones ? 1.0f : scale;
+  __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * s, acc.y * s), hi = __floats2bfloat162_rn(acc.z * s, acc.w * s);
+  uint2 o = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+  // cols is a multiple of 8 and col a multiple of 4: the 4 columns are all inside or all outside
+  if (is_ones) {
+    if (ones_out) *reinterpret_cast<uint2*>(ones_out + n0 + col) = o;
+  } else {
+    *reinterpret_cast<uint2*>(out + j * p.cols + n0 + col) = o;
   }
 }
 
