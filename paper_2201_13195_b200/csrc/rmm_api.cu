@@ -42,10 +42,10 @@ Workspace workspace_layout(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rm
   w.scratch_off = off;
   size_t scratch = (size_t)w.db_slices * (size_t)D_out * sizeof(float);
   if (dt == RMM_DTYPE_BF16) {
-    const tc::SketchSchedule f = tc::make_sketch_schedule(k, D_in, N, tc::SK_MAX_CTAS);
-    const tc::SketchSchedule b = tc::make_sketch_schedule(k + 1, D_out, N, tc::SK_MAX_CTAS);
-    const long long slots = f.num_slots() > b.num_slots() ? f.num_slots() : b.num_slots();
-    scratch = (size_t)slots * tc::SK_TILE_ELEMS * sizeof(float);
+    // an upper bound over every grid the launch may use: one partial tile per (tile, CTA) pair at most
+    const long long tf = ((k + tc::SK_BM - 1) / tc::SK_BM) * ((D_in + tc::SK_BN - 1) / tc::SK_BN);
+    const long long tb = ((k + 1 + tc::SK_BM - 1) / tc::SK_BM) * ((D_out + tc::SK_BN - 1) / tc::SK_BN);
+    scratch = (size_t)((tf > tb ? tf : tb) + tc::SK_MAX_CTAS) * tc::SK_TILE_ELEMS * sizeof(float);
   }
   off += align_up(scratch);
   w.total = off;
@@ -61,11 +61,30 @@ struct DeviceState {
   bool ok = false;
   EncodeTiledFn encode = nullptr;
   int num_sms = 0;
+  int sketch_clusters[5] = {0, 0, 0, 0, 0};   // [C]: clusters of C CTAs of the sketch kernel resident at once
 };
 
 template <typename K>
 bool allow_big_smem(K kernel, int bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+// How many clusters of `c` CTAs of kernel `k` can be resident on the device at once.
+template <typename K>
+bool query_clusters(K k, int c, int* out) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3((unsigned)(tc::SK_MAX_CTAS / c * c));
+  cfg.blockDim = dim3(tc::SK_THREADS);
+  cfg.dynamicSmemBytes = tc::SK_SMEM_BYTES;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, k, &cfg) != cudaSuccess || n < 1) return false;
+  *out = n < tc::SK_MAX_CTAS / c ? n : tc::SK_MAX_CTAS / c;
+  return true;
 }
 
 DeviceState& device_state() {
@@ -88,7 +107,14 @@ DeviceState& device_state() {
     a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_K>, tc::GEMM_SMEM_BYTES);
     a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_MN>, tc::GEMM_SMEM_BYTES);
     a &= allow_big_smem(tc::gemm_kernel<tc::A_MN, tc::B_MN>, tc::GEMM_SMEM_BYTES);
-    a &= allow_big_smem(tc::sketch_kernel, tc::SK_SMEM_BYTES);
+    a &= allow_big_smem(tc::sketch_kernel<1>, tc::SK_SMEM_BYTES);
+    a &= allow_big_smem(tc::sketch_kernel<2>, tc::SK_SMEM_BYTES);
+    a &= allow_big_smem(tc::sketch_kernel<4>, tc::SK_SMEM_BYTES);
+    if (a) {
+      st.sketch_clusters[1] = st.num_sms < tc::SK_MAX_CTAS ? st.num_sms : tc::SK_MAX_CTAS;
+      a &= query_clusters(tc::sketch_kernel<2>, 2, &st.sketch_clusters[2]);
+      a &= query_clusters(tc::sketch_kernel<4>, 4, &st.sketch_clusters[4]);
+    }
     st.ok = a;
   });
   return st;
@@ -172,10 +198,23 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   p.dist = dist;
   p.ones_row = ones_out ? 1 : 0;
   p.status = status;
-  const int sms = device_state().num_sms;
-  p.sched = tc::make_sketch_schedule(p.rows, cols, tokens, sms < tc::SK_MAX_CTAS ? sms : tc::SK_MAX_CTAS);
-  tc::sketch_kernel<<<p.sched.num_ctas, tc::SK_THREADS, tc::SK_SMEM_BYTES, stream>>>(tmB, p, pk);
-  dim3 rgrid((unsigned)p.sched.tiles(), tc::SK_BM);
+  const int C = tc::sketch_cluster_size(cols);
+  p.sched = tc::make_sketch_schedule(p.rows, cols, tokens, C, device_state().sketch_clusters[C]);
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3((unsigned)(C * p.sched.num_ctas));      // the schedule's workers are clusters
+  cfg.blockDim = dim3(tc::SK_THREADS);
+  cfg.dynamicSmemBytes = tc::SK_SMEM_BYTES;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t le = C == 4 ? cudaLaunchKernelEx(&cfg, tc::sketch_kernel<4>, tmB, p, pk)
+                 : C == 2 ? cudaLaunchKernelEx(&cfg, tc::sketch_kernel<2>, tmB, p, pk)
+                          : cudaLaunchKernelEx(&cfg, tc::sketch_kernel<1>, tmB, p, pk);
+  if (le != cudaSuccess) return RMM_ERR_CUDA;
+  dim3 rgrid((unsigned)(p.sched.tiles() * C), tc::SK_BM);
   tc::sketch_reduce_kernel<<<rgrid, 128, 0, stream>>>(p, c, reinterpret_cast<__nv_bfloat16*>(out),
                                                       reinterpret_cast<__nv_bfloat16*>(ones_out));
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
@@ -386,9 +425,10 @@ rmm_status rmm_debug_gauss_words(const uint32_t* words, int64_t n, float* out, v
 int64_t rmm_debug_sketch_schedule(int64_t rows, int64_t cols, int64_t tokens, int max_ctas, int mode, int64_t* records,
                                   int64_t cap, int64_t* info) {
   if (rows < 1 || cols < 1 || tokens < 1 || max_ctas < 1) return -1;
-  const tc::SketchSchedule sc = tc::make_sketch_schedule(rows, cols, tokens, max_ctas);
+  const int C = tc::sketch_cluster_size(cols);
+  const tc::SketchSchedule sc = tc::make_sketch_schedule(rows, cols, tokens, C, max_ctas / C > 0 ? max_ctas / C : 1);
   if (info) {
-    info[0] = sc.tiles(); info[1] = sc.ksteps; info[2] = sc.num_ctas; info[3] = sc.num_slots();
+    info[0] = sc.tiles(); info[1] = sc.ksteps; info[2] = sc.num_ctas; info[3] = sc.num_slots(); info[4] = C;
   }
   int64_t n = 0;
   auto put = [&](int64_t a, int64_t b, int64_t c, int64_t d, int64_t e) {

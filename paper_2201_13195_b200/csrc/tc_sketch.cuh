@@ -7,19 +7,32 @@
 //
 // Work decomposition.  An output tile is 128 sketch rows x 512 columns: the whole tensor
 // memory of an SM (512 fp32 columns) accumulates it, so that every generated entry of S
-// is used 512 times.  There are far fewer such tiles than SMs and each has a long
-// contraction (all tokens), so the (tile, 64-token step) units are laid out in one line
-// and cut into equal contiguous ranges, one per CTA.  A CTA accumulates each of the (at
-// most a few) tile segments in its range in tensor memory and writes it as an fp32
-// partial tile; sketch_reduce_kernel adds the partial tiles of every output tile in a
-// fixed order, applies the scale c = 1/sqrt(B_proj) (Eq. 5) and rounds to bf16.
+// is used 512 times by the CTA that holds it.
+//
+// Sharing S across a cluster.  Generating the normals is plain ALU work (about 29
+// instructions each) and would cost more time than the MMAs that consume them.  CTAs that
+// compute the same sketch rows for neighbouring 512-column blocks therefore form a
+// thread-block cluster of C (1, 2 or 4): each CTA generates 128/C rows of every S^T stage and
+// stores them, with ordinary distributed-shared-memory stores, into the operand ring of
+// all C CTAs, so each generated entry feeds C x 512 columns.  Every CTA runs its own
+// TMA ring for its B columns, its own MMAs and its own accumulator.
+//
+// Stream-K.  There are far fewer tiles than SMs and each has a long contraction (all tokens),
+// so (tile group, 64-token step) units are distributed over the clusters by a static
+// schedule (below).  A CTA accumulates each tile segment of its cluster's share in tensor
+// memory and writes it as an fp32 partial tile; sketch_reduce_kernel adds the partial tiles
+// of every output tile in a fixed order, applies the scale c = 1/sqrt(B_proj) (Eq. 5) and
+// rounds to bf16.
 //
 // db for free: when ones_row is set, row index B_proj of S^T is a row of ones, so row
 // B_proj of the result is sum_n dY[n][:] (Eq. 3); the reduce kernel stores it, unscaled.
 //
 // Warp roles: warp 0 TMA producer (B), warp 1 tensor-memory owner and MMA issuer, warps
 // 2..17 generate S tiles and drain the accumulator.  A stages hold 64 tokens, B stages 32
-// tokens (so that four of each fit in shared memory); all waits are bounded.
+// tokens.  Barriers of a CTA: fullA[s] (C x generating warps: the stage is complete in this
+// CTA's ring), emptyA[s] (C commits: every CTA of the cluster has consumed the stage, so it
+// may be overwritten everywhere), fullB / emptyB (TMA ring), accfull / accempty.  All waits
+// are bounded.
 #pragma once
 #include "sketch_rng.cuh"
 #include "tc_common.cuh"
@@ -37,10 +50,12 @@ constexpr int SK_GEN_THREADS = 32 * SK_GEN_WARPS;
 constexpr int SK_THREADS = 64 + SK_GEN_THREADS;
 constexpr int SK_SMEM_BYTES = SK_A_STAGES * SK_A_BYTES + SK_B_STAGES * SK_B_BYTES + 1024 + 256;
 constexpr int SK_TILE_ELEMS = SK_BM * SK_BN;         // fp32 elements of one partial tile
-constexpr int SK_MAX_CTAS = 148;                     // grid size used for workspace sizing
+constexpr int SK_MAX_CTAS = 148;                     // CTAs (all clusters together) used for workspace sizing
 
 // Static schedule shared by the sketch kernel, the reduce kernel and the host.
 //
+// A "tile" of the schedule is a tile group: 128 rows x (C x 512) columns, worked on by one
+// cluster of C CTAs; "CTA" below means one such cluster.
 // Units are (tile, 64-token step) pairs; every CTA gets `upc` consecutive units of a
 // line that is ordered so that CTAs running at the same time read the same token rows
 // of B (they then come out of L2 instead of being fetched from HBM once per tile row):
@@ -52,8 +67,9 @@ constexpr int SK_MAX_CTAS = 148;                     // grid size used for works
 //      into ranges of `upc` units, which may span several tiles.
 // Every (CTA, tile) intersection is one segment = one fp32 partial tile (slot).
 struct SketchSchedule {
-  int tiles_m, tiles_n, ksteps;
-  int num_ctas;            // grid size
+  int cluster;             // C: CTAs per cluster = 512-column blocks per tile group
+  int tiles_m, tiles_n, ksteps;   // tiles_n counts tile groups
+  int num_ctas;            // number of clusters
   int rounds;              // whole-tile rounds
   int tiles_rem;           // tiles handled by the blocked part
   int upc;                 // units per CTA in the blocked part
@@ -150,10 +166,18 @@ __host__ __device__ inline void sketch_for_each_slot_of_tile(const SketchSchedul
 
 inline long long gcd_ll(long long a, long long b) { while (b) { long long t = a % b; a = b; b = t; } return a; }
 
-inline SketchSchedule make_sketch_schedule(long long rows, long long cols, long long tokens, int max_ctas) {
+// Cluster size for a result with `cols` columns: the largest of 4, 2, 1 that divides the number
+// of 512-column blocks.
+inline int sketch_cluster_size(long long cols) {
+  const long long blocks = (cols + SK_BN - 1) / SK_BN;
+  return blocks % 2 == 0 ? 2 : 1;
+}
+
+inline SketchSchedule make_sketch_schedule(long long rows, long long cols, long long tokens, int cluster, int max_ctas) {
   SketchSchedule s;
+  s.cluster = cluster;
   s.tiles_m = (int)((rows + SK_BM - 1) / SK_BM);
-  s.tiles_n = (int)((cols + SK_BN - 1) / SK_BN);
+  s.tiles_n = (int)((cols + (long long)SK_BN * cluster - 1) / ((long long)SK_BN * cluster));
   s.ksteps = (int)((tokens + SK_AK - 1) / SK_AK);
   const int tiles = s.tiles_m * s.tiles_n;
   s.rounds = tiles / max_ctas;
@@ -185,6 +209,36 @@ struct SketchParams {
   int* status;
   SketchSchedule sched;
 };
+
+// Eight consecutive tokens (tok8 a multiple of 8) of sketch row j as packed bf16: one 16-byte
+// chunk of the operand tile.
+__device__ __forceinline__ uint4 sketch_chunk(const PhiloxKey& pk, const SketchParams& p, long long j, long long tok8) {
+  constexpr uint32_t kOnes = 0x3f803f80u;   // two bf16 1.0
+  uint4 v;
+  if (p.dist == 0) {
+    v = gaussian_8_bf16(pk, (uint32_t)tok8, (uint32_t)j);
+  } else if (p.dist == 1) {
+    uint32_t w[4];
+    rademacher_128(pk, (uint32_t)(tok8 >> 7), (uint32_t)j, w);
+    const int t = (int)(tok8 & 127);
+    uint32_t word = w[0];                    // select without dynamic indexing
+    word = (t >> 5) == 1 ? w[1] : word;
+    word = (t >> 5) == 2 ? w[2] : word;
+    word = (t >> 5) == 3 ? w[3] : word;
+    v = rademacher_8_bf16(word, (t & 31) >> 3);
+  } else {
+    const long long d = j - tok8;
+    uint32_t q0 = 0, q1 = 0, q2 = 0, q3 = 0;
+    if (d >= 0 && d < 8) {
+      const uint32_t one = (d & 1) ? 0x3f800000u : 0x00003f80u;
+      const int wi = (int)(d >> 1);
+      q0 = wi == 0 ? one : 0u; q1 = wi == 1 ? one : 0u; q2 = wi == 2 ? one : 0u; q3 = wi == 3 ? one : 0u;
+    }
+    v = make_uint4(q0, q1, q2, q3);
+  }
+  if (p.ones_row && j == p.b_proj) v = make_uint4(kOnes, kOnes, kOnes, kOnes);
+  return v;
+}
 
 // One 128 x 64 stage of S^T, K-major with the 128-byte swizzle: row r at byte 128 r, its
 // 16-byte chunk c (tokens 8c .. 8c+7) stored at chunk position c ^ (r & 7).
@@ -233,6 +287,7 @@ __device__ __forceinline__ void sketch_generate_stage(uint8_t* a_tile, const Phi
   }
 }
 
+template <int C>
 __global__ void __launch_bounds__(SK_THREADS, 1)
 sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey pk) {
   extern __shared__ uint8_t smem_raw[];
@@ -250,14 +305,21 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * SK_A_STAGES + 2 * SK_B_STAGES + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+  // tasks = (row, 16-byte chunk) pairs of a stage; this CTA generates rows [rank*128/C, (rank+1)*128/C)
+  constexpr int TASKS = SK_BM * 8 / C;                                         // per CTA and stage
+  constexpr int GEN_ACTIVE_THREADS = TASKS < SK_GEN_THREADS ? TASKS : SK_GEN_THREADS;
+  constexpr int GEN_ACTIVE_WARPS = GEN_ACTIVE_THREADS / 32;
+  constexpr int TASKS_PER_THREAD = TASKS / GEN_ACTIVE_THREADS;
+
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = (C == 1) ? 0u : cluster_ctarank();
   const SketchSchedule& sc = p.sched;
-  const int cta = (int)blockIdx.x;
+  const int cl = (int)(blockIdx.x / C);          // cluster index = worker index of the schedule
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < SK_A_STAGES; ++s) {
-      mbar_init(fulla_bar(s), SK_GEN_WARPS);      // one arrival per generator warp
-      mbar_init(emptya_bar(s), 1);
+      mbar_init(fulla_bar(s), C * GEN_ACTIVE_WARPS);
+      mbar_init(emptya_bar(s), C);
     }
     for (int s = 0; s < SK_B_STAGES; ++s) {
       mbar_init(fullb_bar(s), 1);
@@ -273,12 +335,12 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     tmem_relinquish();
   }
   tc_fence_before();
-  __syncthreads();
+  if (C == 1) __syncthreads(); else cluster_sync_all();   // every CTA's barriers exist before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer (B)
+    // ------------------------------------------------------------ TMA producer (this CTA's B columns)
     if (lane == 0) {
       tma_prefetch_desc(&tmB);
       int s = 0;
@@ -287,8 +349,8 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       int seg_it = 0;
       long long cursor = 0;
       SketchSegment sg;
-      while (ok && sketch_next_segment(sc, cta, seg_it, cursor, sg)) {
-        const int n0 = (sg.tile % sc.tiles_n) * SK_BN;
+      while (ok && sketch_next_segment(sc, cl, seg_it, cursor, sg)) {
+        const int n0 = ((sg.tile % sc.tiles_n) * C + (int)rank) * SK_BN;
         for (int ks = sg.ks0; ks < sg.ks1 && ok; ++ks) {
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
@@ -313,6 +375,9 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       // added to the start-address field (16-byte units).
       const uint64_t adesc0 = smem_desc_sw128(smem_u32(a_ring), 16, 1024);
       const uint64_t bdesc0 = smem_desc_sw128(smem_u32(b_ring), SK_B_SLAB, 1024);
+      uint32_t peer_emptya0[C];                  // emptyA[0] of every CTA of the cluster
+#pragma unroll
+      for (int r = 0; r < C; ++r) peer_emptya0[r] = (C == 1) ? emptya_bar(0) : mapa_shared(emptya_bar(0), r);
       int sa = 0, sb = 0;
       uint32_t pha = 0, phb = 0;
       int seg = 0;
@@ -320,7 +385,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       int seg_it = 0;
       long long cursor = 0;
       SketchSegment sg;
-      for (; ok && sketch_next_segment(sc, cta, seg_it, cursor, sg); ++seg) {
+      for (; ok && sketch_next_segment(sc, cl, seg_it, cursor, sg); ++seg) {
         if (seg > 0) {   // the previous segment's accumulator must have been drained
           ok = mbar_wait(accempty_bar, (uint32_t)(seg - 1) & 1u, abort_flag, p.status);
           if (!ok) break;
@@ -328,8 +393,10 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
         }
         uint32_t acc = 0;
         for (int ks = sg.ks0; ks < sg.ks1 && ok; ++ks) {
-          ok = mbar_wait(fulla_bar(sa), pha, abort_flag, p.status);
+          ok = (C == 1) ? mbar_wait(fulla_bar(sa), pha, abort_flag, p.status)
+                        : mbar_wait_cluster(fulla_bar(sa), pha, abort_flag, p.status);
           if (!ok) break;
+          if (C > 1) fence_proxy_async_smem();   // stage written by generic stores of the whole cluster
           const uint64_t ad = adesc0 + (uint64_t)(sa * (SK_A_BYTES >> 4));
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
@@ -348,7 +415,11 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
             umma_commit(emptyb_bar(sb));
             if (++sb == SK_B_STAGES) { sb = 0; phb ^= 1u; }
           }
-          if (ok) umma_commit(emptya_bar(sa));
+          if (ok) {
+            // tell every CTA of the cluster (all of them write into this stage) that this CTA is done with it
+#pragma unroll
+            for (int r = 0; r < C; ++r) umma_commit(peer_emptya0[r] + 8u * sa);
+          }
           if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
         }
         if (ok) umma_commit(accfull_bar);
@@ -359,6 +430,14 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     // ------------------------------------------------------------ S generators + accumulator drain
     const int gtid = threadIdx.x - 64;
     const int gw = warp - 2;
+    const bool gen_active = gtid < GEN_ACTIVE_THREADS;
+    uint32_t ring_base[C];                       // a_ring of every CTA of the cluster
+    uint32_t peer_fulla0 = 0;                    // lane r < C: fullA[0] of CTA r
+    if (C > 1) {
+#pragma unroll
+      for (int r = 0; r < C; ++r) ring_base[r] = mapa_shared(smem_u32(a_ring), r);
+      if (lane < C) peer_fulla0 = mapa_shared(fulla_bar(0), lane);
+    }
     int sa = 0;
     uint32_t pha = 0;
     int seg = 0;
@@ -366,16 +445,37 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     int seg_it = 0;
     long long cursor = 0;
     SketchSegment sg;
-    for (; ok && sketch_next_segment(sc, cta, seg_it, cursor, sg); ++seg) {
+    for (; ok && sketch_next_segment(sc, cl, seg_it, cursor, sg); ++seg) {
       const int tile = sg.tile;
       const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
-      for (int ks = sg.ks0; ks < sg.ks1; ++ks) {
-        if (!mbar_wait(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        sketch_generate_stage(a_ring + sa * SK_A_BYTES, pk, p, m0, (long long)ks * SK_AK, gtid);
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(fulla_bar(sa));
-        if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
+      if (gen_active) {
+        for (int ks = sg.ks0; ks < sg.ks1; ++ks) {
+          const bool freed = (C == 1) ? mbar_wait(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)
+                                      : mbar_wait_cluster(emptya_bar(sa), pha ^ 1u, abort_flag, p.status);
+          if (!freed) { ok = false; break; }
+          if (C == 1) {
+            sketch_generate_stage(a_ring + sa * SK_A_BYTES, pk, p, m0, (long long)ks * SK_AK, gtid);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(fulla_bar(sa));
+          } else {
+            // this CTA's rows of the stage, stored into every CTA's ring
+#pragma unroll
+            for (int it = 0; it < TASKS_PER_THREAD; ++it) {
+              const int t = it * GEN_ACTIVE_THREADS + gtid;
+              const int r = (int)rank * (SK_BM / C) + (t >> 3), c = t & 7;
+              const uint4 v = sketch_chunk(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
+              const uint32_t off = (uint32_t)(sa * SK_A_BYTES + r * 128 + ((c ^ (r & 7)) << 4));
+#pragma unroll
+              for (int q = 0; q < C; ++q) st_shared_cluster_v4(ring_base[q] + off, v);
+            }
+            // no proxy fence here: the release below publishes the warp's stores to the cluster, and
+            // the MMA issuer of each CTA fences generic -> async after it has acquired the stage
+            __syncwarp();
+            if (lane < C) mbar_arrive_cluster(peer_fulla0 + 8u * sa);
+          }
+          if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
+        }
       }
       ok = __all_sync(0xffffffffu, ok && mbar_wait(accfull_bar, (uint32_t)seg & 1u, abort_flag, p.status));
       if (!ok) break;
@@ -383,7 +483,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       {
         const int q = warp & 3;                 // tensor-memory lane quarter of this warp
         const int cgroup = gw >> 2;             // 4 warps share a quarter: 128 columns each
-        float* slot = p.partial + sg.slot * (long long)SK_TILE_ELEMS;
+        float* slot = p.partial + (sg.slot * C + rank) * (long long)SK_TILE_ELEMS;
         float* prow = slot + (long long)(q * 32 + lane) * SK_BN;
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
@@ -408,19 +508,21 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     while (clock64() - t0 < 2000000ll) __nanosleep(1000);
   }
   tc_fence_before();
-  __syncthreads();
+  if (C == 1) __syncthreads(); else cluster_sync_all();   // nobody leaves while a neighbour may still store or signal here
   if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
 // Adds the partial tiles of each output tile in schedule order, scales, rounds to bf16.
-// grid = (tiles, 128 rows), block = 128 threads: thread t owns columns 4t .. 4t+3 of one row.
+// grid = (tile groups * C, 128 rows), block = 128 threads: thread t owns columns 4t .. 4t+3 of one
+// row; blockIdx.x = C * tile group + rank of the CTA that produced the 512-column block.
 // All loads of a thread are independent, so the kernel runs at memory speed.
 constexpr int SKR_MAX_SLOTS = 8;     // partial tiles summed per batch of loads
 __global__ void __launch_bounds__(128)
 sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ ones_out) {
   const SketchSchedule& sc = p.sched;
-  const int tile = blockIdx.x;
-  const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM, n0 = (long long)(tile % sc.tiles_n) * SK_BN;
+  const int tile = blockIdx.x / sc.cluster, rank = blockIdx.x % sc.cluster;
+  const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
+  const long long n0 = ((long long)(tile % sc.tiles_n) * sc.cluster + rank) * SK_BN;
   const int r = blockIdx.y;
   const long long j = m0 + r;
   const int col = threadIdx.x * 4;
@@ -433,7 +535,7 @@ sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ ou
     float4 v[SKR_MAX_SLOTS];
 #pragma unroll
     for (int i = 0; i < SKR_MAX_SLOTS; ++i)
-      if (i < ns) v[i] = __ldcs(reinterpret_cast<const float4*>(p.partial + slots[i] * (long long)SK_TILE_ELEMS + off));
+      if (i < ns) v[i] = __ldcs(reinterpret_cast<const float4*>(p.partial + (slots[i] * sc.cluster + rank) * (long long)SK_TILE_ELEMS + off));
 #pragma unroll
     for (int i = 0; i < SKR_MAX_SLOTS; ++i)
       if (i < ns) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
