@@ -64,7 +64,8 @@ constexpr int SK_MAX_CTAS = 148;                     // CTAs (all clusters toget
 //      block b of tile t goes to CTA b * tiles_rem + t, so all CTAs of a block walk the
 //      same token range in step;
 //   3. the last, narrower block (width `w_last`) is laid out tile after tile and cut
-//      into ranges of `upc` units, which may span several tiles.
+//      into ranges of `upc` units, which may span several tiles -- unless that would give a
+//      CTA many short segments, in which case the tiles are cut into equal blocks only.
 // Every (CTA, tile) intersection is one segment = one fp32 partial tile (slot).
 struct SketchSchedule {
   int cluster;             // C: CTAs per cluster = 512-column blocks per tile group
@@ -118,7 +119,8 @@ __host__ __device__ inline bool sketch_next_segment(const SketchSchedule& sc, in
     if (it > sc.rounds) return false;
     const int b = cta / sc.tiles_rem, t = cta % sc.tiles_rem;
     seg.tile = base_tile + t;
-    seg.ks0 = b * sc.upc; seg.ks1 = seg.ks0 + sc.upc;
+    seg.ks0 = b * sc.upc;
+    seg.ks1 = seg.ks0 + sc.upc < sc.ksteps ? seg.ks0 + sc.upc : sc.ksteps;   // the last block may be narrower
     seg.slot = sc.slot_block(b, t);
     ++it;
     return true;
@@ -190,6 +192,22 @@ inline SketchSchedule make_sketch_schedule(long long rows, long long cols, long 
     if (s.upc < 4 && s.upc < s.ksteps) s.upc = s.ksteps < 4 ? s.ksteps : 4;   // no slivers
     s.full_blocks = s.ksteps / s.upc;
     s.w_last = s.ksteps - s.full_blocks * s.upc;
+    if (s.w_last > 0 && s.full_blocks > 0) {
+      // A narrow last block gives a few CTAs many short segments, each of which costs a drain of
+      // the accumulator (about kSegCost steps' worth).  Compare with cutting every tile into
+      // full_blocks equal blocks instead (fewer CTAs busy, one segment each) and take the
+      // schedule whose busiest CTA finishes first.
+      constexpr int kSegCost = 8;
+      const int segs_last = (s.upc + s.w_last - 1) / s.w_last + 1;
+      const int cost_stream = s.upc + kSegCost * segs_last;
+      const int upc_even = (s.ksteps + s.full_blocks - 1) / s.full_blocks;
+      const int cost_even = upc_even + kSegCost;
+      if (cost_even <= cost_stream) {
+        s.upc = upc_even;
+        s.full_blocks = (s.ksteps + s.upc - 1) / s.upc;
+        s.w_last = 0;
+      }
+    }
     if (s.w_last > 0) s.lcm_last = (long long)s.upc / gcd_ll(s.upc, s.w_last) * s.w_last;
     const long long last_ctas = s.w_last > 0 ? ((long long)s.tiles_rem * s.w_last + s.upc - 1) / s.upc : 0;
     const long long used = (long long)s.full_blocks * s.tiles_rem + last_ctas;
