@@ -61,6 +61,7 @@ struct DeviceState {
   bool ok = false;
   EncodeTiledFn encode = nullptr;
   int num_sms = 0;
+  int gemm_pairs = 0;                         // CTA pairs of the GEMM kernel resident at once
   int sketch_clusters[5] = {0, 0, 0, 0, 0};   // [C]: clusters of C CTAs of the sketch kernel resident at once
 };
 
@@ -71,14 +72,14 @@ bool allow_big_smem(K kernel, int bytes) {
 
 // How many clusters of `c` CTAs of kernel `k` can be resident on the device at once.
 template <typename K>
-bool query_clusters(K k, int c, int* out) {
+bool query_clusters(K k, int c, int* out, int threads = tc::SK_THREADS, int smem = tc::SK_SMEM_BYTES) {
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.gridDim = dim3((unsigned)(tc::SK_MAX_CTAS / c * c));
-  cfg.blockDim = dim3(tc::SK_THREADS);
-  cfg.dynamicSmemBytes = tc::SK_SMEM_BYTES;
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.dynamicSmemBytes = (size_t)smem;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n = 0;
@@ -113,6 +114,7 @@ DeviceState& device_state() {
     if (a) {
       st.sketch_clusters[1] = st.num_sms < tc::SK_MAX_CTAS ? st.num_sms : tc::SK_MAX_CTAS;
       a &= query_clusters(tc::sketch_kernel<2>, 2, &st.sketch_clusters[2]);
+      a &= query_clusters(tc::gemm_kernel<tc::A_K, tc::B_K>, 2, &st.gemm_pairs, 64 + 32 * tc::NEPI, tc::GEMM_SMEM_BYTES);
       a &= query_clusters(tc::sketch_kernel<4>, 4, &st.sketch_clusters[4]);
     }
     st.ok = a;
@@ -170,16 +172,25 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   bool ok = true;
   if (AMODE == tc::A_K) ok &= make_tmap(&tmA, a, M, K, tc::BM);
   if (AMODE == tc::A_MN) ok &= make_tmap(&tmA, a, K, M, tc::BK);
-  if (BMODE == tc::B_K) ok &= make_tmap(&tmB, b, N, K, tc::BN);
+  if (BMODE == tc::B_K) ok &= make_tmap(&tmB, b, N, K, tc::BN_HALF);
   if (BMODE == tc::B_MN) ok &= make_tmap(&tmB, b, K, N, tc::BK);
   if (!ok) return RMM_ERR_CUDA;
   tc::GemmParams p;
   p.M = M; p.N = N; p.K = K;
   p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.status = status;
-  const int64_t tiles = ((N + tc::BN - 1) / tc::BN) * ((M + tc::BM - 1) / tc::BM);
-  const int sms = device_state().num_sms;
-  dim3 grid((unsigned)(tiles < sms ? tiles : sms));   // persistent: one CTA per SM
-  tc::gemm_kernel<AMODE, BMODE><<<grid, 64 + 32 * tc::NEPI, tc::GEMM_SMEM_BYTES, stream>>>(tmA, tmB, p);
+  const int64_t tiles = ((N + tc::BN - 1) / tc::BN) * ((M + tc::PAIR_M - 1) / tc::PAIR_M);
+  const int max_pairs = device_state().gemm_pairs;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(2 * (unsigned)(tiles < max_pairs ? tiles : max_pairs));   // persistent CTA pairs
+  cfg.blockDim = dim3(64 + 32 * tc::NEPI);
+  cfg.dynamicSmemBytes = tc::GEMM_SMEM_BYTES;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, tc::gemm_kernel<AMODE, BMODE>, tmA, tmB, p) != cudaSuccess) return RMM_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
 

@@ -1,5 +1,5 @@
 // Tensor-core contraction kernel for the bf16 mode (sm_100a): C = alpha * A B^T (+ bias),
-// bf16 operands, fp32 accumulation in tensor memory, 128 x 256 output tiles, persistent CTAs.
+// bf16 operands, fp32 accumulation in tensor memory, persistent CTA pairs.
 //
 // The three dense contractions of Algorithm 1 whose operands all live in memory differ only
 // in the operand layouts (the two sketch contractions are in tc_sketch.cuh):
@@ -10,24 +10,35 @@
 // "MN-major" operands are consumed in place through the transpose bits of the tcgen05
 // instruction descriptor; nothing is transposed in memory.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = tensor-memory owner and MMA issuer,
-// warps 2..5 = epilogue.  Stages of a ring of shared-memory buffers are handed over with
-// mbarriers: full (TMA bytes landed), empty (tcgen05.commit: the MMAs that read the stage
-// have retired), accfull (all MMAs of the tile retired), accempty (the epilogue has read the
-// accumulator buffer out of tensor memory).
+// CTA pairs.  Two CTAs on neighbouring SMs (a cluster of two) compute one 256 x 256 output tile
+// with tcgen05.mma.cta_group::2: each CTA stages its own 128 rows of A and only half (128) of
+// the tile's B columns, the hardware feeds both halves of B to both tensor cores, and each CTA
+// keeps the 128 x 256 accumulator of its rows in its own tensor memory.  Per MMA this halves
+// the B bytes an SM pulls from L2 and pushes through its shared memory, which is what limits a
+// one-CTA 128 x 256 tile, and it makes room for six pipeline stages instead of four.
+//
+// Warp roles per CTA: warp 0 = TMA producer (its halves), warp 1 = tensor-memory owner and, in
+// the leader CTA (even rank), MMA issuer; warps 2..5 = epilogue.  Barriers: full (leader; TMA
+// bytes of both CTAs landed), empty (both; tcgen05.commit from the leader: the MMAs that read
+// the stage have retired), accfull (both; all MMAs of the tile retired), accempty (leader; the
+// epilogues of both CTAs have read the accumulator buffer out of tensor memory).  Two
+// accumulator buffers: the MMAs of tile i+1 overlap the epilogue of tile i.
 #pragma once
 #include "tc_common.cuh"
 
 namespace rmm {
 namespace tc {
 
-constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
-constexpr int STAGES = 4;
+constexpr int BM = 128;                       // rows of A (and of the accumulator) per CTA
+constexpr int PAIR_M = 2 * BM;                // rows of a pair tile
+constexpr int BN = 256, BK = 64, UMMA_K = 16;
+constexpr int BN_HALF = BN / 2;               // B columns staged by each CTA
+constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2;          // 16 KiB
-constexpr int B_BYTES = BN * BK * 2;          // 32 KiB
+constexpr int B_BYTES = BN_HALF * BK * 2;     // 16 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SLAB_BYTES = 64 * BK * 2;       // one [64 k][64 mn] MN-major slab, 8 KiB
-constexpr int TMEM_COLS = 512;              // two 128 x 256 fp32 accumulators: MMAs of tile i+1 overlap the epilogue of tile i
+constexpr int TMEM_COLS = 512;                // two 128 x 256 fp32 accumulators per CTA
 constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 enum : int { A_K = 0, A_MN = 1 };
@@ -65,11 +76,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // Persistent: this CTA takes tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Tile t is
-  // (m = t / tiles_n, n = t % tiles_n): the CTAs of one wave share a few A row blocks (the large,
+  const uint32_t rank = cluster_ctarank();       // 0 = leader of the pair
+  const bool leader = rank == 0;
+  // Persistent: this pair takes pair tiles pair, pair + num_pairs, ...  Tile t is
+  // (m = t / tiles_n, n = t % tiles_n): the pairs of one wave share a few A row blocks (the large,
   // token-sized operand is then read from HBM once) and sweep all of B (weights, L2 resident).
+  const int pair = (int)(blockIdx.x >> 1), num_pairs = (int)(gridDim.x >> 1);
   const int tiles_n = (int)((p.N + BN - 1) / BN);
-  const int num_tiles = (int)((p.M + BM - 1) / BM) * tiles_n;
+  const int num_tiles = (int)((p.M + PAIR_M - 1) / PAIR_M) * tiles_n;
   const int num_kb = (int)((p.K + BK - 1) / BK);
 
   if (threadIdx.x == 0) {
@@ -79,46 +93,51 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(accfull_bar(b), 1);
-      mbar_init(accempty_bar(b), NEPI);     // one arrival per epilogue warp
+      mbar_init(accempty_bar(b), 2 * NEPI);     // one arrival per epilogue warp of either CTA
     }
     *abort_flag = 0;
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
-    tmem_relinquish();
+    tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+    tmem_relinquish_pair();
   }
   tc_fence_before();
-  __syncthreads();
+  cluster_sync_all();      // both CTAs' barriers and tensor memory exist before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------ TMA producer: this CTA's halves
     if (lane == 0) {
       tma_prefetch_desc(&tmA);
       tma_prefetch_desc(&tmB);
+      const uint32_t leader_delta = mapa_shared(bar0, 0) - bar0;   // 0 in the leader itself
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+        const int m0 = (tile / tiles_n) * PAIR_M + (int)rank * BM;
+        const int n0 = (tile % tiles_n) * BN + (int)rank * BN_HALF;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          if (!mbar_wait_cluster(empty_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t a_smem = sbase + s * STAGE_BYTES, b_smem = a_smem + A_BYTES;
-          mbar_arrive_expect_tx(full_bar(s), A_BYTES + B_BYTES);
+          if (leader) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);   // bytes of both CTAs
+          const uint32_t full_leader = full_bar(s) + leader_delta;
           const int k0 = kb * BK;
           if (AMODE == A_K) {
-            tma_load_2d(a_smem, &tmA, full_bar(s), k0, m0);
+            tma_load_2d_pair(a_smem, &tmA, full_leader, k0, m0);
           } else {
 #pragma unroll
-            for (int sl = 0; sl < BM / 64; ++sl) tma_load_2d(a_smem + sl * SLAB_BYTES, &tmA, full_bar(s), m0 + 64 * sl, k0);
+            for (int sl = 0; sl < BM / 64; ++sl)
+              tma_load_2d_pair(a_smem + sl * SLAB_BYTES, &tmA, full_leader, m0 + 64 * sl, k0);
           }
           if (BMODE == B_K) {
-            tma_load_2d(b_smem, &tmB, full_bar(s), k0, n0);
+            tma_load_2d_pair(b_smem, &tmB, full_leader, k0, n0);
           } else {
 #pragma unroll
-            for (int sl = 0; sl < BN / 64; ++sl) tma_load_2d(b_smem + sl * SLAB_BYTES, &tmB, full_bar(s), n0 + 64 * sl, k0);
+            for (int sl = 0; sl < BN_HALF / 64; ++sl)
+              tma_load_2d_pair(b_smem + sl * SLAB_BYTES, &tmB, full_leader, n0 + 64 * sl, k0);
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
@@ -126,40 +145,46 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc_bf16(BM, BN, AMODE == A_MN, BMODE == B_MN);
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16(PAIR_M, BN, AMODE == A_MN, BMODE == B_MN);
       // Descriptors are built once; a stage or K step only adds to the 14-bit start-address
-      // field (16-byte units), which never carries out of it.
+      // field (16-byte units), which never carries out of it.  The same shared-memory offsets
+      // are used in both CTAs.
       const uint64_t adesc0 = (AMODE == A_MN) ? smem_desc_sw128(sbase, SLAB_BYTES, 1024) : smem_desc_sw128(sbase, 16, 1024);
       const uint64_t bdesc0 = (BMODE == B_MN) ? smem_desc_sw128(sbase + A_BYTES, SLAB_BYTES, 1024)
                                               : smem_desc_sw128(sbase + A_BYTES, 16, 1024);
       constexpr uint32_t a_kstep = ((AMODE == A_MN) ? UMMA_K * 128 : UMMA_K * 2) >> 4;
       constexpr uint32_t b_kstep = ((BMODE == B_MN) ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+      const uint32_t peer_delta = mapa_shared(bar0, 1) - bar0;
       bool ok = true;
       int s = 0;
       uint32_t ph = 0;
-      int it = 0;                               // tiles done by this CTA
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+      int it = 0;                               // tiles done by this pair
+      for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++it) {
         const int buf = it & 1;
-        // the epilogue must have drained this accumulator buffer (two tiles ago)
-        ok = mbar_wait(accempty_bar(buf), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, p.status);
+        // the epilogues of both CTAs must have drained this accumulator buffer (two tiles ago)
+        ok = mbar_wait_cluster(accempty_bar(buf), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
+          ok = mbar_wait_cluster(full_bar(s), ph, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
           const uint64_t ad = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
           const uint64_t bd = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
 #pragma unroll
           for (int j = 0; j < BK / UMMA_K; ++j)
-            umma_bf16(d_tmem, ad + j * a_kstep, bd + j * b_kstep, idesc, (kb | j) != 0 ? 1u : 0u);
-          umma_commit(empty_bar(s));
+            umma_bf16_pair(d_tmem, ad + j * a_kstep, bd + j * b_kstep, idesc, (kb | j) != 0 ? 1u : 0u);
+          umma_commit_pair(empty_bar(s));
+          umma_commit_pair(empty_bar(s) + peer_delta);
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
-        if (ok) umma_commit(accfull_bar(buf));
+        if (ok) {
+          umma_commit_pair(accfull_bar(buf));
+          umma_commit_pair(accfull_bar(buf) + peer_delta);
+        }
       }
     }
     __syncwarp();
@@ -167,14 +192,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ------------------------------------------------------------ epilogue (overlaps the next tile's MMAs)
     const int q = warp & 3;                       // tensor-memory lane quarter this warp may read
     const __nv_bfloat16* bias = reinterpret_cast<const __nv_bfloat16*>(p.bias);
+    const uint32_t accempty_leader0 = mapa_shared(accempty_bar(0), 0);
     int it = 0;
-    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+    for (int tile = pair; tile < num_tiles; tile += num_pairs, ++it) {
       const int buf = it & 1;
       const bool acc_ready =
-          __all_sync(0xffffffffu, mbar_wait(accfull_bar(buf), (uint32_t)(it >> 1) & 1u, abort_flag, p.status));
+          __all_sync(0xffffffffu, mbar_wait_cluster(accfull_bar(buf), (uint32_t)(it >> 1) & 1u, abort_flag, p.status));
       if (!acc_ready) break;
       tc_fence_after();
-      const int64_t m0 = (int64_t)(tile / tiles_n) * BM, n0 = (int64_t)(tile % tiles_n) * BN;
+      const int64_t m0 = (int64_t)(tile / tiles_n) * PAIR_M + (int64_t)rank * BM, n0 = (int64_t)(tile % tiles_n) * BN;
       const int64_t row = m0 + q * 32 + lane;
       __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc;
 #pragma unroll 1
@@ -209,10 +235,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
         }
       }
-      // hand the buffer back to the MMA issuer
+      // hand the buffer back to the MMA issuer in the leader CTA
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(accempty_bar(buf));
+      if (lane == 0) mbar_arrive_cluster(accempty_leader0 + 8u * buf);
     }
   }
   // ---------------------------------------------------------------- teardown
@@ -222,8 +248,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     while (clock64() - t0 < 2000000ll) __nanosleep(1000);
   }
   tc_fence_before();
-  __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+  cluster_sync_all();      // nobody leaves while its partner may still signal or read across
+  if (warp == 1) tmem_dealloc_pair(tmem_base, TMEM_COLS);
 }
 
 }  // namespace tc
