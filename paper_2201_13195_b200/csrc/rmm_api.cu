@@ -134,6 +134,20 @@ bool make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, i
                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of a row-major bf16 matrix [rows][cols], cols a multiple of 64, viewed as
+// (column in slab: 64, row, slab: cols / 64); box = [box_slabs][box_rows][64]: in shared memory the
+// slabs ([box_rows][64 columns], 128-byte swizzle) follow one another, which is the MN-major
+// operand layout, and one TMA instruction fetches all of them.  Rows out of range read as zero.
+bool make_tmap_slabs(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows, int box_slabs) {
+  cuuint64_t gdim[3] = {64u, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+  cuuint64_t gstride[2] = {(cuuint64_t)cols * 2, 128u};
+  cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, (cuuint32_t)box_slabs};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  return device_state().encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstride, box,
+                               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // ------------------------------------------------------------------ per-kernel timing (benchmarks)
 struct ProfileRecord { int step; cudaEvent_t t0, t1; };
 struct Profiler {
@@ -199,8 +213,12 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
 rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, int64_t cols, int64_t tokens, float c,
                          int dist, const PhiloxKey& pk, float* partial, int* status, cudaStream_t stream) {
   CUtensorMap tmB;
-  if (!make_tmap(&tmB, b, tokens, cols, tc::SK_BK)) return RMM_ERR_CUDA;
+  const bool slab_map = cols % 64 == 0;
+  if (!(slab_map ? make_tmap_slabs(&tmB, b, tokens, cols, tc::SK_BK, tc::SK_BN / 64)
+                 : make_tmap(&tmB, b, tokens, cols, tc::SK_BK)))
+    return RMM_ERR_CUDA;
   tc::SketchParams p;
+  p.slab_map = slab_map ? 1 : 0;
   p.rows = k + (ones_out ? 1 : 0);
   p.b_proj = k;
   p.cols = cols;

@@ -224,6 +224,7 @@ struct SketchParams {
   float* partial;      // [num_slots][128][512] fp32
   int dist;
   int ones_row;
+  int slab_map;        // tmB is the 3-D (column in slab, token, slab) view: needs cols % 64 == 0
   int* status;
   SketchSchedule sched;
 };
@@ -258,52 +259,8 @@ __device__ __forceinline__ uint4 sketch_chunk(const PhiloxKey& pk, const SketchP
   return v;
 }
 
-// One 128 x 64 stage of S^T, K-major with the 128-byte swizzle: row r at byte 128 r, its
-// 16-byte chunk c (tokens 8c .. 8c+7) stored at chunk position c ^ (r & 7).
-__device__ __forceinline__ void sketch_generate_stage(uint8_t* a_tile, const PhiloxKey& pk, const SketchParams& p,
-                                                      long long m0, long long n0, int gtid) {
-  constexpr uint32_t kOnes = 0x3f803f80u;   // two bf16 1.0
-  if (p.dist == 0) {
-#pragma unroll
-    for (int it = 0; it < (SK_BM * 8) / SK_GEN_THREADS; ++it) {
-      const int t = it * SK_GEN_THREADS + gtid;
-      const int r = t >> 3, c = t & 7;
-      uint4 v = gaussian_8_bf16(pk, (uint32_t)(n0 + 8 * c), (uint32_t)(m0 + r));
-      if (p.ones_row && m0 + r == p.b_proj) v = make_uint4(kOnes, kOnes, kOnes, kOnes);
-      *reinterpret_cast<uint4*>(a_tile + r * 128 + ((c ^ (r & 7)) << 4)) = v;
-    }
-  } else if (p.dist == 1) {
-    // one thread per (row, 16 tokens): 2 chunks out of one Philox word
-    const int r = gtid >> 2, h = gtid & 3;
-    uint32_t w[4];
-    rademacher_128(pk, (uint32_t)(n0 >> 7), (uint32_t)(m0 + r), w);
-    const uint32_t word = w[((n0 & 127) >> 5) + (h >> 1)];
-    const bool ones = p.ones_row && m0 + r == p.b_proj;
-#pragma unroll
-    for (int b = 0; b < 2; ++b) {
-      const int c = 2 * h + b;
-      uint4 v = rademacher_8_bf16(word, 2 * (h & 1) + b);
-      if (ones) v = make_uint4(kOnes, kOnes, kOnes, kOnes);
-      *reinterpret_cast<uint4*>(a_tile + r * 128 + ((c ^ (r & 7)) << 4)) = v;
-    }
-  } else {
-#pragma unroll
-    for (int it = 0; it < (SK_BM * 8) / SK_GEN_THREADS; ++it) {
-      const int t = it * SK_GEN_THREADS + gtid;
-      const int r = t >> 3, c = t & 7;
-      const long long d = (m0 + r) - (n0 + 8 * c);
-      uint32_t q0 = 0, q1 = 0, q2 = 0, q3 = 0;
-      if (d >= 0 && d < 8) {
-        const uint32_t one = (d & 1) ? 0x3f800000u : 0x00003f80u;
-        const int wi = (int)(d >> 1);
-        q0 = wi == 0 ? one : 0u; q1 = wi == 1 ? one : 0u; q2 = wi == 2 ? one : 0u; q3 = wi == 3 ? one : 0u;
-      }
-      uint4 v = make_uint4(q0, q1, q2, q3);
-      if (p.ones_row && m0 + r == p.b_proj) v = make_uint4(kOnes, kOnes, kOnes, kOnes);
-      *reinterpret_cast<uint4*>(a_tile + r * 128 + ((c ^ (r & 7)) << 4)) = v;
-    }
-  }
-}
+// Layout of an S^T stage (128 rows x 64 tokens): K-major with the 128-byte swizzle: row r at
+// byte 128 r, its 16-byte chunk c (tokens 8c .. 8c+7) stored at chunk position c ^ (r & 7).
 
 template <int C>
 __global__ void __launch_bounds__(SK_THREADS, 1)
@@ -376,9 +333,14 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
             const uint32_t b_smem = smem_u32(b_ring) + s * SK_B_BYTES;
             mbar_arrive_expect_tx(fullb_bar(s), SK_B_BYTES);
             const int tok0 = ks * SK_AK + half * SK_BK;
+            if (p.slab_map) {
+              // one instruction for all eight [32 tokens][64 columns] slabs of the stage
+              tma_load_3d(b_smem, &tmB, fullb_bar(s), 0, tok0, n0 >> 6);
+            } else {
 #pragma unroll
-            for (int sl = 0; sl < SK_BN / 64; ++sl)
-              tma_load_2d(b_smem + sl * SK_B_SLAB, &tmB, fullb_bar(s), n0 + 64 * sl, tok0);
+              for (int sl = 0; sl < SK_BN / 64; ++sl)
+                tma_load_2d(b_smem + sl * SK_B_SLAB, &tmB, fullb_bar(s), n0 + 64 * sl, tok0);
+            }
             if (++s == SK_B_STAGES) { s = 0; ph ^= 1u; }
           }
         }
@@ -468,25 +430,33 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
       if (gen_active) {
         for (int ks = sg.ks0; ks < sg.ks1; ++ks) {
+          // Generate first, into registers: the normals do not depend on the ring, so the wait for
+          // a free stage only covers the stores.
+          uint4 v[TASKS_PER_THREAD];
+          uint32_t off[TASKS_PER_THREAD];
+#pragma unroll
+          for (int it = 0; it < TASKS_PER_THREAD; ++it) {
+            const int t = it * GEN_ACTIVE_THREADS + gtid;
+            const int r = (int)rank * (SK_BM / C) + (t >> 3), c = t & 7;
+            v[it] = sketch_chunk(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
+            off[it] = (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+          }
           const bool freed = (C == 1) ? mbar_wait(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)
                                       : mbar_wait_cluster(emptya_bar(sa), pha ^ 1u, abort_flag, p.status);
           if (!freed) { ok = false; break; }
           if (C == 1) {
-            sketch_generate_stage(a_ring + sa * SK_A_BYTES, pk, p, m0, (long long)ks * SK_AK, gtid);
+#pragma unroll
+            for (int it = 0; it < TASKS_PER_THREAD; ++it)
+              *reinterpret_cast<uint4*>(a_ring + sa * SK_A_BYTES + off[it]) = v[it];
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(fulla_bar(sa));
           } else {
             // this CTA's rows of the stage, stored into every CTA's ring
 #pragma unroll
-            for (int it = 0; it < TASKS_PER_THREAD; ++it) {
-              const int t = it * GEN_ACTIVE_THREADS + gtid;
-              const int r = (int)rank * (SK_BM / C) + (t >> 3), c = t & 7;
-              const uint4 v = sketch_chunk(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
-              const uint32_t off = (uint32_t)(sa * SK_A_BYTES + r * 128 + ((c ^ (r & 7)) << 4));
+            for (int it = 0; it < TASKS_PER_THREAD; ++it)
 #pragma unroll
-              for (int q = 0; q < C; ++q) st_shared_cluster_v4(ring_base[q] + off, v);
-            }
+              for (int q = 0; q < C; ++q) st_shared_cluster_v4(ring_base[q] + sa * SK_A_BYTES + off[it], v[it]);
             // no proxy fence here: the release below publishes the warp's stores to the cluster, and
             // the MMA issuer of each CTA fences generic -> async after it has acquired the stage
             __syncwarp();
