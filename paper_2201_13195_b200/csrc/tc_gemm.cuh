@@ -146,7 +146,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
-    if (leader && lane == 0) {
+    // The whole warp runs the loop, so that descriptors and addresses stay warp-uniform (the
+    // tcgen05 operands live in uniform registers); one elected lane issues.
+    if (leader) {
       constexpr uint32_t idesc = instr_desc_bf16(PAIR_M, BN, AMODE == A_MN, BMODE == B_MN);
       // Descriptors are built once; a stage or K step only adds to the 14-bit start-address
       // field (16-byte units), which never carries out of it.  The same shared-memory offsets
@@ -164,26 +166,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++it) {
         const int buf = it & 1;
         // the epilogues of both CTAs must have drained this accumulator buffer (two tiles ago)
-        ok = mbar_wait_cluster(accempty_bar(buf), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, p.status);
+        ok = (mbar_wait_cluster_warp(accempty_bar(buf), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, p.status));
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = mbar_wait_cluster(full_bar(s), ph, abort_flag, p.status);
+          ok = (mbar_wait_cluster_warp(full_bar(s), ph, abort_flag, p.status));
           if (!ok) break;
           tc_fence_after();
           const uint64_t ad = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
           const uint64_t bd = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
+          if (elect_one()) {
 #pragma unroll
-          for (int j = 0; j < BK / UMMA_K; ++j)
-            umma_bf16_pair(d_tmem, ad + j * a_kstep, bd + j * b_kstep, idesc, (kb | j) != 0 ? 1u : 0u);
-          umma_commit_pair(empty_bar(s));
-          umma_commit_pair(empty_bar(s) + peer_delta);
+            for (int j = 0; j < BK / UMMA_K; ++j)
+              umma_bf16_pair(d_tmem, ad + j * a_kstep, bd + j * b_kstep, idesc, (kb | j) != 0 ? 1u : 0u);
+            umma_commit_pair(empty_bar(s));
+            umma_commit_pair(empty_bar(s) + peer_delta);
+          }
+          __syncwarp();
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (ok) {
-          umma_commit_pair(accfull_bar(buf));
-          umma_commit_pair(accfull_bar(buf) + peer_delta);
+          if (elect_one()) {
+            umma_commit_pair(accfull_bar(buf));
+            umma_commit_pair(accfull_bar(buf) + peer_delta);
+          }
+          __syncwarp();
         }
       }
     }
@@ -197,7 +205,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     for (int tile = pair; tile < num_tiles; tile += num_pairs, ++it) {
       const int buf = it & 1;
       const bool acc_ready =
-          __all_sync(0xffffffffu, mbar_wait_cluster(accfull_bar(buf), (uint32_t)(it >> 1) & 1u, abort_flag, p.status));
+          (mbar_wait_cluster_warp(accfull_bar(buf), (uint32_t)(it >> 1) & 1u, abort_flag, p.status));
       if (!acc_ready) break;
       tc_fence_after();
       const int64_t m0 = (int64_t)(tile / tiles_n) * PAIR_M + (int64_t)rank * BM, n0 = (int64_t)(tile % tiles_n) * BN;

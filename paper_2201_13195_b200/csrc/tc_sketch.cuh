@@ -349,10 +349,12 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp runs the loop, so that descriptors and addresses stay warp-uniform (the
+    // tcgen05 operands live in uniform registers); one elected lane issues.
+    {
       constexpr uint32_t idesc = instr_desc_bf16(SK_BM, 256, false, true);
-      // One thread issues everything: descriptors are built once, stage and K-step offsets are
-      // added to the start-address field (16-byte units).
+      // Descriptors are built once, stage and K-step offsets are added to the start-address
+      // field (16-byte units).
       const uint64_t adesc0 = smem_desc_sw128(smem_u32(a_ring), 16, 1024);
       const uint64_t bdesc0 = smem_desc_sw128(smem_u32(b_ring), SK_B_SLAB, 1024);
       uint32_t peer_emptya0[C];                  // emptyA[0] of every CTA of the cluster
@@ -367,42 +369,51 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       SketchSegment sg;
       for (; ok && sketch_next_segment(sc, cl, seg_it, cursor, sg); ++seg) {
         if (seg > 0) {   // the previous segment's accumulator must have been drained
-          ok = mbar_wait(accempty_bar, (uint32_t)(seg - 1) & 1u, abort_flag, p.status);
+          ok = (mbar_wait_warp(accempty_bar, (uint32_t)(seg - 1) & 1u, abort_flag, p.status));
           if (!ok) break;
           tc_fence_after();
         }
         uint32_t acc = 0;
         for (int ks = sg.ks0; ks < sg.ks1 && ok; ++ks) {
-          ok = (C == 1) ? mbar_wait(fulla_bar(sa), pha, abort_flag, p.status)
-                        : mbar_wait_cluster(fulla_bar(sa), pha, abort_flag, p.status);
+          ok = (C == 1) ? mbar_wait_warp(fulla_bar(sa), pha, abort_flag, p.status)
+                        : mbar_wait_cluster_warp(fulla_bar(sa), pha, abort_flag, p.status);
           if (!ok) break;
           if (C > 1) fence_proxy_async_smem();   // stage written by generic stores of the whole cluster
           const uint64_t ad = adesc0 + (uint64_t)(sa * (SK_A_BYTES >> 4));
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            ok = mbar_wait(fullb_bar(sb), phb, abort_flag, p.status);
+            ok = (mbar_wait_warp(fullb_bar(sb), phb, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
             const uint64_t bd = bdesc0 + (uint64_t)(sb * (SK_B_BYTES >> 4));
+            if (elect_one()) {
 #pragma unroll
-            for (int j = 0; j < SK_BK / 16; ++j) {
+              for (int j = 0; j < SK_BK / 16; ++j) {
 #pragma unroll
-              for (int nh = 0; nh < 2; ++nh)
-                umma_bf16(tmem_base + nh * 256, ad + (half * (SK_BK / 16) + j) * 2,
-                          bd + ((nh * 4 * SK_B_SLAB + j * 2048) >> 4), idesc, acc);
-              acc = 1;
+                for (int nh = 0; nh < 2; ++nh)
+                  umma_bf16(tmem_base + nh * 256, ad + (half * (SK_BK / 16) + j) * 2,
+                            bd + ((nh * 4 * SK_B_SLAB + j * 2048) >> 4), idesc, (acc | (uint32_t)j) != 0 ? 1u : 0u);
+              }
+              umma_commit(emptyb_bar(sb));
             }
-            umma_commit(emptyb_bar(sb));
+            __syncwarp();
+            acc = 1;
             if (++sb == SK_B_STAGES) { sb = 0; phb ^= 1u; }
           }
           if (ok) {
             // tell every CTA of the cluster (all of them write into this stage) that this CTA is done with it
+            if (elect_one()) {
 #pragma unroll
-            for (int r = 0; r < C; ++r) umma_commit(peer_emptya0[r] + 8u * sa);
+              for (int r = 0; r < C; ++r) umma_commit(peer_emptya0[r] + 8u * sa);
+            }
+            __syncwarp();
           }
           if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
         }
-        if (ok) umma_commit(accfull_bar);
+        if (ok) {
+          if (elect_one()) umma_commit(accfull_bar);
+          __syncwarp();
+        }
       }
     }
     __syncwarp();
@@ -441,8 +452,8 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
             v[it] = sketch_chunk(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
             off[it] = (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
           }
-          const bool freed = (C == 1) ? mbar_wait(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)
-                                      : mbar_wait_cluster(emptya_bar(sa), pha ^ 1u, abort_flag, p.status);
+          const bool freed = (C == 1) ? mbar_wait_warp(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)
+                                      : mbar_wait_cluster_warp(emptya_bar(sa), pha ^ 1u, abort_flag, p.status);
           if (!freed) { ok = false; break; }
           if (C == 1) {
 #pragma unroll
@@ -465,7 +476,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
           if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
         }
       }
-      ok = __all_sync(0xffffffffu, ok && mbar_wait(accfull_bar, (uint32_t)seg & 1u, abort_flag, p.status));
+      ok = ok && mbar_wait_warp(accfull_bar, (uint32_t)seg & 1u, abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();
       {
@@ -508,7 +519,8 @@ constexpr int SKR_MAX_SLOTS = 8;     // partial tiles summed per batch of loads
 __global__ void __launch_bounds__(128)
 sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ ones_out) {
   const SketchSchedule& sc = p.sched;
-  const int tile = blockIdx.x / sc.cluster, rank = blockIdx.x % sc.cluster;
+  const int per_tile = sc.cluster;      // partial tiles (CTAs) per schedule tile
+  const int tile = blockIdx.x / per_tile, rank = blockIdx.x % per_tile;
   const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
   const long long n0 = ((long long)(tile % sc.tiles_n) * sc.cluster + rank) * SK_BN;
   const int r = blockIdx.y;
@@ -523,7 +535,7 @@ sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ ou
     float4 v[SKR_MAX_SLOTS];
 #pragma unroll
     for (int i = 0; i < SKR_MAX_SLOTS; ++i)
-      if (i < ns) v[i] = __ldcs(reinterpret_cast<const float4*>(p.partial + (slots[i] * sc.cluster + rank) * (long long)SK_TILE_ELEMS + off));
+      if (i < ns) v[i] = __ldcs(reinterpret_cast<const float4*>(p.partial + (slots[i] * per_tile + rank) * (long long)SK_TILE_ELEMS + off));
 #pragma unroll
     for (int i = 0; i < SKR_MAX_SLOTS; ++i)
       if (i < ns) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
