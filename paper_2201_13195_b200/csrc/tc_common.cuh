@@ -103,6 +103,14 @@ __device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint
                "r"(v.w)
                : "memory");
 }
+// 16-byte asynchronous store into the shared memory of any CTA of the cluster; its completion is
+// counted (16 bytes) on an mbarrier of that same CTA, so the consumer's wait on the barrier
+// covers the data and no release fence is needed on the producer side.
+__device__ __forceinline__ void st_async_cluster_v4(uint32_t cluster_addr, uint4 v, uint32_t cluster_mbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(cluster_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(cluster_mbar)
+               : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(

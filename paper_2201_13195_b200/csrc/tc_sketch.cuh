@@ -293,7 +293,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < SK_A_STAGES; ++s) {
-      mbar_init(fulla_bar(s), C * GEN_ACTIVE_WARPS);
+      mbar_init(fulla_bar(s), C == 1 ? GEN_ACTIVE_WARPS : 1);   // C > 1: one local arrival + the bytes of the stage
       mbar_init(emptya_bar(s), C);
     }
     for (int s = 0; s < SK_B_STAGES; ++s) {
@@ -378,7 +378,6 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
           ok = (C == 1) ? mbar_wait_warp(fulla_bar(sa), pha, abort_flag, p.status)
                         : mbar_wait_cluster_warp(fulla_bar(sa), pha, abort_flag, p.status);
           if (!ok) break;
-          if (C > 1) fence_proxy_async_smem();   // stage written by generic stores of the whole cluster
           const uint64_t ad = adesc0 + (uint64_t)(sa * (SK_A_BYTES >> 4));
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
@@ -387,6 +386,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
             tc_fence_after();
             const uint64_t bd = bdesc0 + (uint64_t)(sb * (SK_B_BYTES >> 4));
             if (elect_one()) {
+              if (C > 1 && half == 0) fence_proxy_async_smem();   // stage stored by other threads of the cluster
 #pragma unroll
               for (int j = 0; j < SK_BK / 16; ++j) {
 #pragma unroll
@@ -423,11 +423,13 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     const int gw = warp - 2;
     const bool gen_active = gtid < GEN_ACTIVE_THREADS;
     uint32_t ring_base[C];                       // a_ring of every CTA of the cluster
-    uint32_t peer_fulla0 = 0;                    // lane r < C: fullA[0] of CTA r
+    uint32_t peer_fulla[C];                      // fullA[0] of every CTA of the cluster
     if (C > 1) {
 #pragma unroll
-      for (int r = 0; r < C; ++r) ring_base[r] = mapa_shared(smem_u32(a_ring), r);
-      if (lane < C) peer_fulla0 = mapa_shared(fulla_bar(0), lane);
+      for (int r = 0; r < C; ++r) {
+        ring_base[r] = mapa_shared(smem_u32(a_ring), r);
+        peer_fulla[r] = mapa_shared(fulla_bar(0), r);
+      }
     }
     int sa = 0;
     uint32_t pha = 0;
@@ -463,15 +465,15 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
             __syncwarp();
             if (lane == 0) mbar_arrive(fulla_bar(sa));
           } else {
-            // this CTA's rows of the stage, stored into every CTA's ring
+            // This CTA's rows of the stage go into every CTA's ring as asynchronous stores that
+            // count their bytes on the destination's fullA barrier; the barrier completes when all
+            // 16 KiB of the stage (from all C CTAs) have landed and the local arrival below is in.
+            if (gtid == 0) mbar_arrive_expect_tx(fulla_bar(sa), SK_A_BYTES);
 #pragma unroll
             for (int it = 0; it < TASKS_PER_THREAD; ++it)
 #pragma unroll
-              for (int q = 0; q < C; ++q) st_shared_cluster_v4(ring_base[q] + sa * SK_A_BYTES + off[it], v[it]);
-            // no proxy fence here: the release below publishes the warp's stores to the cluster, and
-            // the MMA issuer of each CTA fences generic -> async after it has acquired the stage
-            __syncwarp();
-            if (lane < C) mbar_arrive_cluster(peer_fulla0 + 8u * sa);
+              for (int q = 0; q < C; ++q)
+                st_async_cluster_v4(ring_base[q] + sa * SK_A_BYTES + off[it], v[it], peer_fulla[q] + 8u * sa);
           }
           if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
         }
