@@ -45,6 +45,7 @@ constexpr int SK_A_STAGES = 4, SK_B_STAGES = 4;
 constexpr int SK_A_BYTES = SK_BM * SK_AK * 2;        // 16 KiB
 constexpr int SK_B_BYTES = SK_BN * SK_BK * 2;        // 32 KiB
 constexpr int SK_B_SLAB = 64 * SK_BK * 2;            // [32 tokens][64 columns] = 4 KiB
+constexpr int SK_STAGGER = 2;                        // steps by which neighbouring tile rows are offset
 constexpr int SK_GEN_WARPS = 16;
 constexpr int SK_GEN_THREADS = 32 * SK_GEN_WARPS;
 constexpr int SK_THREADS = 64 + SK_GEN_THREADS;
@@ -94,6 +95,17 @@ struct SketchSchedule {
     return (long long)rounds * num_ctas + (long long)full_blocks * tiles_rem + ci + t - seg_start / lcm_last;
   }
 };
+
+// Token step visited at position i of a segment.  Segments of different tile rows start at
+// different offsets (and wrap around), so that the CTAs that walk the same token range do not all
+// ask L2 for the same rows of B at the same moment.  The sum of a segment does not depend on the
+// order of its steps up to fp32 rounding, and the order is a fixed function of the schedule.
+__host__ __device__ inline int sketch_step(int ks0, int ks1, int tile_m, int i) {
+  const int len = ks1 - ks0;
+  int k = i + (tile_m * SK_STAGGER) % len;
+  if (k >= len) k -= len;
+  return ks0 + k;
+}
 
 // One segment of work of a CTA.
 struct SketchSegment {
@@ -326,7 +338,8 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       SketchSegment sg;
       while (ok && sketch_next_segment(sc, cl, seg_it, cursor, sg)) {
         const int n0 = ((sg.tile % sc.tiles_n) * C + (int)rank) * SK_BN;
-        for (int ks = sg.ks0; ks < sg.ks1 && ok; ++ks) {
+        for (int i = 0; i < sg.ks1 - sg.ks0 && ok; ++i) {
+          const int ks = sketch_step(sg.ks0, sg.ks1, sg.tile / sc.tiles_n, i);
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             if (!mbar_wait(emptyb_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
@@ -442,7 +455,8 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       const int tile = sg.tile;
       const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
       if (gen_active) {
-        for (int ks = sg.ks0; ks < sg.ks1; ++ks) {
+        for (int i = 0; i < sg.ks1 - sg.ks0; ++i) {
+          const int ks = sketch_step(sg.ks0, sg.ks1, tile / sc.tiles_n, i);
           // Generate first, into registers: the normals do not depend on the ring, so the wait for
           // a free stage only covers the stores.
           uint4 v[TASKS_PER_THREAD];
