@@ -22,11 +22,6 @@ constexpr uint32_t kWaitLimitPolls = 1u << 30;
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile(
@@ -76,6 +71,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// Early test of a barrier phase ("peek").  A barrier test is a long round trip for the one warp
+// that issues MMAs; started one stage ahead, it overlaps the MMA issue of the current stage, and
+// the blocking wait is only entered when the early test said "not yet".  The predicate lives in
+// a PTX register that MBAR_PEEK_DECLARE() declares once, in the entry block of the kernel;
+// slot is a literal 0 or 1.  All lanes of the warp test the same address in one instruction, so
+// they read the same answer.
+#define MBAR_PEEK_DECLARE() asm volatile(".reg .pred mbar_peek0, mbar_peek1;")
+#define MBAR_PEEK(slot, bar, parity) \
+  asm volatile("mbarrier.test_wait.parity.shared::cta.b64 mbar_peek" #slot ", [%0], %1;" ::"r"(bar), "r"(parity) : "memory")
+#define MBAR_PEEK_CLUSTER(slot, bar, parity)                                                                       \
+  asm volatile("mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 mbar_peek" #slot ", [%0], %1;" ::"r"(bar), \
+               "r"(parity)                                                                                          \
+               : "memory")
+#define MBAR_PEEK_RESULT(slot, out) asm volatile("selp.u32 %0, 1, 0, mbar_peek" #slot ";" : "=r"(out)::"memory")
+
 // ---------------------------------------------------------------- thread-block clusters
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -97,18 +107,15 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-// 16-byte store into the shared memory of any CTA of the cluster (distributed shared memory)
-__device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint4 v) {
-  asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(v.x), "r"(v.y), "r"(v.z),
-               "r"(v.w)
-               : "memory");
-}
-// 16-byte asynchronous store into the shared memory of any CTA of the cluster; its completion is
-// counted (16 bytes) on an mbarrier of that same CTA, so the consumer's wait on the barrier
-// covers the data and no release fence is needed on the producer side.
-__device__ __forceinline__ void st_async_cluster_v4(uint32_t cluster_addr, uint4 v, uint32_t cluster_mbar) {
-  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
-               ::"r"(cluster_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(cluster_mbar)
+// Asynchronous copy of `bytes` (a multiple of 16, both addresses 16-byte aligned) from this CTA's
+// shared memory into the shared memory of a CTA of the cluster (address from mapa_shared). The
+// bytes are counted on an mbarrier of the destination CTA, so the consumer's wait on that barrier
+// covers the data. The source is read through the async proxy: writers fence with
+// fence_proxy_async_smem() before the issuing thread is told that the data is there.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster_addr, uint32_t src_cta_addr, uint32_t bytes,
+                                                     uint32_t cluster_mbar) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_cluster_addr), "r"(src_cta_addr), "r"(bytes), "r"(cluster_mbar)
                : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
@@ -187,11 +194,6 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc,
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr)
                : "memory");
-}
-
-// generic-proxy writes into shared memory of the cluster -> visible to the async proxy there
-__device__ __forceinline__ void fence_proxy_async_smem_cluster() {
-  asm volatile("fence.proxy.async.shared::cluster;" ::: "memory");
 }
 
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA, tcgen05)

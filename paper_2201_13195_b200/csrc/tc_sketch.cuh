@@ -48,7 +48,8 @@ constexpr int SK_B_SLAB = 64 * SK_BK * 2;            // [32 tokens][64 columns] 
 constexpr int SK_STAGGER = 2;                        // steps by which neighbouring tile rows are offset
 constexpr int SK_GEN_WARPS = 16;
 constexpr int SK_GEN_THREADS = 32 * SK_GEN_WARPS;
-constexpr int SK_THREADS = 64 + SK_GEN_THREADS;
+constexpr int SK_MMA_WARPS = 2;            // each issues the MMAs of one 256-column half of the tile
+constexpr int SK_THREADS = 32 * (1 + SK_MMA_WARPS) + SK_GEN_THREADS;
 constexpr int SK_SMEM_BYTES = SK_A_STAGES * SK_A_BYTES + SK_B_STAGES * SK_B_BYTES + 1024 + 256;
 constexpr int SK_TILE_ELEMS = SK_BM * SK_BN;         // fp32 elements of one partial tile
 constexpr int SK_MAX_CTAS = 148;                     // CTAs (all clusters together) used for workspace sizing
@@ -291,13 +292,19 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
   const uint32_t accempty_bar = accfull_bar + 8u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * SK_A_STAGES + 2 * SK_B_STAGES + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint32_t* gen_count = tmem_slot + 2;           // generator warps that have stored their part of a stage
 
-  // tasks = (row, 16-byte chunk) pairs of a stage; this CTA generates rows [rank*128/C, (rank+1)*128/C)
+  // tasks = (row, 16-byte chunk) pairs of a stage; this CTA generates rows [rank*128/C, (rank+1)*128/C).
+  // The generator warps form one group per ring stage: group g fills stage g of the ring, i.e.
+  // the K-steps g, g + 4, ... of this CTA's sequence.  The groups run out of phase, so the stores,
+  // fences and barrier round trips of one group are covered by the arithmetic of the others.
   constexpr int TASKS = SK_BM * 8 / C;                                         // per CTA and stage
-  constexpr int GEN_ACTIVE_THREADS = TASKS < SK_GEN_THREADS ? TASKS : SK_GEN_THREADS;
-  constexpr int GEN_ACTIVE_WARPS = GEN_ACTIVE_THREADS / 32;
-  constexpr int TASKS_PER_THREAD = TASKS / GEN_ACTIVE_THREADS;
+  constexpr int GROUP_WARPS = SK_GEN_WARPS / SK_A_STAGES;
+  constexpr int GROUP_THREADS = 32 * GROUP_WARPS;
+  constexpr int TASKS_PER_THREAD = TASKS / GROUP_THREADS;
+  static_assert(SK_GEN_WARPS % SK_A_STAGES == 0 && TASKS % GROUP_THREADS == 0, "generator groups");
 
+  MBAR_PEEK_DECLARE();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = (C == 1) ? 0u : cluster_ctarank();
   const SketchSchedule& sc = p.sched;
@@ -305,14 +312,15 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < SK_A_STAGES; ++s) {
-      mbar_init(fulla_bar(s), C == 1 ? GEN_ACTIVE_WARPS : 1);   // C > 1: one local arrival + the bytes of the stage
-      mbar_init(emptya_bar(s), C);
+      mbar_init(fulla_bar(s), GROUP_WARPS);   // C > 1: plus the bytes that the other CTAs copy in
+      mbar_init(emptya_bar(s), C * SK_MMA_WARPS);
+      gen_count[s] = 0;
     }
     for (int s = 0; s < SK_B_STAGES; ++s) {
       mbar_init(fullb_bar(s), 1);
-      mbar_init(emptyb_bar(s), 1);
+      mbar_init(emptyb_bar(s), SK_MMA_WARPS);
     }
-    mbar_init(accfull_bar, 1);
+    mbar_init(accfull_bar, SK_MMA_WARPS);
     mbar_init(accempty_bar, SK_GEN_WARPS);
     *abort_flag = 0;
     fence_barrier_init();
@@ -360,8 +368,13 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
+  } else if (warp <= SK_MMA_WARPS) {
+    // ------------------------------------------------------------ MMA issuers
+    // Two warps, one per 256-column half of the accumulator: the issue loop is a serial chain of
+    // barrier waits, descriptor arithmetic, MMAs and commits, and one warp alone does not get
+    // through a K-step in the time the tensor pipe needs for it.  Both wait on the same full
+    // barriers; a stage is free once both have committed.
+    const int nh = warp - 1;
     // The whole warp runs the loop, so that descriptors and addresses stay warp-uniform (the
     // tcgen05 operands live in uniform registers); one elected lane issues.
     {
@@ -380,6 +393,9 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       int seg_it = 0;
       long long cursor = 0;
       SketchSegment sg;
+      // Each full barrier is tested one stage ahead (slot 0: S^T ring, slot 1: B ring).
+      if (C == 1) { MBAR_PEEK(0, fulla_bar(0), 0u); } else { MBAR_PEEK_CLUSTER(0, fulla_bar(0), 0u); }
+      MBAR_PEEK(1, fullb_bar(0), 0u);
       for (; ok && sketch_next_segment(sc, cl, seg_it, cursor, sg); ++seg) {
         if (seg > 0) {   // the previous segment's accumulator must have been drained
           ok = (mbar_wait_warp(accempty_bar, (uint32_t)(seg - 1) & 1u, abort_flag, p.status));
@@ -388,40 +404,55 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
         }
         uint32_t acc = 0;
         for (int ks = sg.ks0; ks < sg.ks1 && ok; ++ks) {
-          ok = (C == 1) ? mbar_wait_warp(fulla_bar(sa), pha, abort_flag, p.status)
-                        : mbar_wait_cluster_warp(fulla_bar(sa), pha, abort_flag, p.status);
-          if (!ok) break;
+          uint32_t ready;
+          MBAR_PEEK_RESULT(0, ready);
+          if (!__all_sync(0xffffffffu, ready != 0)) {
+            ok = (C == 1) ? mbar_wait_warp(fulla_bar(sa), pha, abort_flag, p.status)
+                          : mbar_wait_cluster_warp(fulla_bar(sa), pha, abort_flag, p.status);
+            if (!ok) break;
+          }
           const uint64_t ad = adesc0 + (uint64_t)(sa * (SK_A_BYTES >> 4));
+          const int sa_next = (sa + 1 == SK_A_STAGES) ? 0 : sa + 1;
+          const uint32_t pha_next = (sa_next == 0) ? (pha ^ 1u) : pha;
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            ok = (mbar_wait_warp(fullb_bar(sb), phb, abort_flag, p.status));
-            if (!ok) break;
+            MBAR_PEEK_RESULT(1, ready);
+            if (!__all_sync(0xffffffffu, ready != 0)) {
+              ok = (mbar_wait_warp(fullb_bar(sb), phb, abort_flag, p.status));
+              if (!ok) break;
+            }
             tc_fence_after();
             const uint64_t bd = bdesc0 + (uint64_t)(sb * (SK_B_BYTES >> 4));
-            if (elect_one()) {
-              if (C > 1 && half == 0) fence_proxy_async_smem();   // stage stored by other threads of the cluster
+            const int sb_next = (sb + 1 == SK_B_STAGES) ? 0 : sb + 1;
+            const uint32_t phb_next = (sb_next == 0) ? (phb ^ 1u) : phb;
+            const bool issuer = elect_one();
+            if (issuer) {
 #pragma unroll
               for (int j = 0; j < SK_BK / 16; ++j) {
-#pragma unroll
-                for (int nh = 0; nh < 2; ++nh)
-                  umma_bf16(tmem_base + nh * 256, ad + (half * (SK_BK / 16) + j) * 2,
-                            bd + ((nh * 4 * SK_B_SLAB + j * 2048) >> 4), idesc, (acc | (uint32_t)j) != 0 ? 1u : 0u);
+                umma_bf16(tmem_base + nh * 256, ad + (half * (SK_BK / 16) + j) * 2,
+                          bd + ((nh * 4 * SK_B_SLAB + j * 2048) >> 4), idesc, (acc | (uint32_t)j) != 0 ? 1u : 0u);
               }
+            }
+            // the tests of the next stages travel while the commits are issued
+            MBAR_PEEK(1, fullb_bar(sb_next), phb_next);
+            if (half == 1) {
+              if (C == 1) { MBAR_PEEK(0, fulla_bar(sa_next), pha_next); } else { MBAR_PEEK_CLUSTER(0, fulla_bar(sa_next), pha_next); }
+            }
+            if (issuer) {
               umma_commit(emptyb_bar(sb));
+              if (half == 1) {
+                // tell every CTA of the cluster (all of them write into this stage) that this CTA is done with it
+#pragma unroll
+                for (int r = 0; r < C; ++r) umma_commit(peer_emptya0[r] + 8u * sa);
+              }
             }
             __syncwarp();
             acc = 1;
-            if (++sb == SK_B_STAGES) { sb = 0; phb ^= 1u; }
+            sb = sb_next;
+            phb = phb_next;
           }
-          if (ok) {
-            // tell every CTA of the cluster (all of them write into this stage) that this CTA is done with it
-            if (elect_one()) {
-#pragma unroll
-              for (int r = 0; r < C; ++r) umma_commit(peer_emptya0[r] + 8u * sa);
-            }
-            __syncwarp();
-          }
-          if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
+          sa = sa_next;
+          pha = pha_next;
         }
         if (ok) {
           if (elect_one()) umma_commit(accfull_bar);
@@ -432,20 +463,23 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     __syncwarp();
   } else {
     // ------------------------------------------------------------ S generators + accumulator drain
-    const int gtid = threadIdx.x - 64;
-    const int gw = warp - 2;
-    const bool gen_active = gtid < GEN_ACTIVE_THREADS;
-    uint32_t ring_base[C];                       // a_ring of every CTA of the cluster
-    uint32_t peer_fulla[C];                      // fullA[0] of every CTA of the cluster
+    const int gw = warp - 1 - SK_MMA_WARPS;
+    const int grp = gw / GROUP_WARPS;            // ring stage that this warp's group fills
+    const int gtid = (gw % GROUP_WARPS) * 32 + lane;   // thread index within the group
+    constexpr uint32_t PART_BYTES = SK_A_BYTES / C;   // this CTA's rows of a stage: one contiguous block
+    const uint32_t stage_smem = smem_u32(a_ring) + grp * SK_A_BYTES;
+    uint8_t* const stage_ptr = a_ring + grp * SK_A_BYTES;
+    uint32_t peer_part[C];                       // where that block goes in stage grp of every CTA of the cluster
+    uint32_t peer_fulla[C];                      // fullA[grp] of every CTA of the cluster
     if (C > 1) {
 #pragma unroll
       for (int r = 0; r < C; ++r) {
-        ring_base[r] = mapa_shared(smem_u32(a_ring), r);
-        peer_fulla[r] = mapa_shared(fulla_bar(0), r);
+        peer_part[r] = mapa_shared(stage_smem + rank * PART_BYTES, r);
+        peer_fulla[r] = mapa_shared(fulla_bar(grp), r);
       }
     }
-    int sa = 0;
-    uint32_t pha = 0;
+    uint32_t pha = 0;                            // parity of the group's stage
+    int step0 = 0;                               // position of the segment's first K-step in this CTA's sequence
     int seg = 0;
     bool ok = true;
     int seg_it = 0;
@@ -454,44 +488,53 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     for (; ok && sketch_next_segment(sc, cl, seg_it, cursor, sg); ++seg) {
       const int tile = sg.tile;
       const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
-      if (gen_active) {
-        for (int i = 0; i < sg.ks1 - sg.ks0; ++i) {
-          const int ks = sketch_step(sg.ks0, sg.ks1, tile / sc.tiles_n, i);
-          // Generate first, into registers: the normals do not depend on the ring, so the wait for
-          // a free stage only covers the stores.
-          uint4 v[TASKS_PER_THREAD];
-          uint32_t off[TASKS_PER_THREAD];
+      const int len = sg.ks1 - sg.ks0;
+      // the group's first step of this segment: the first i with (step0 + i) % stages == grp
+      for (int i = (grp - step0) & (SK_A_STAGES - 1); i < len; i += SK_A_STAGES) {
+        const int ks = sketch_step(sg.ks0, sg.ks1, tile / sc.tiles_n, i);
+        // Generate first, into registers: the entries do not depend on the ring, so the wait for
+        // the free stage only covers the stores.
+        uint4 v[TASKS_PER_THREAD];
+        uint32_t off[TASKS_PER_THREAD];
 #pragma unroll
-          for (int it = 0; it < TASKS_PER_THREAD; ++it) {
-            const int t = it * GEN_ACTIVE_THREADS + gtid;
-            const int r = (int)rank * (SK_BM / C) + (t >> 3), c = t & 7;
-            v[it] = sketch_chunk(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
-            off[it] = (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
-          }
-          const bool freed = (C == 1) ? mbar_wait_warp(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)
-                                      : mbar_wait_cluster_warp(emptya_bar(sa), pha ^ 1u, abort_flag, p.status);
-          if (!freed) { ok = false; break; }
+        for (int it = 0; it < TASKS_PER_THREAD; ++it) {
+          const int t = it * GROUP_THREADS + gtid;
+          const int r = (int)rank * (SK_BM / C) + (t >> 3), c = t & 7;
+          v[it] = sketch_chunk(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
+          off[it] = (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+        }
+        const bool freed = (C == 1) ? mbar_wait_warp(emptya_bar(grp), pha ^ 1u, abort_flag, p.status)
+                                    : mbar_wait_cluster_warp(emptya_bar(grp), pha ^ 1u, abort_flag, p.status);
+        if (!freed) { ok = false; break; }
+#pragma unroll
+        for (int it = 0; it < TASKS_PER_THREAD; ++it) *reinterpret_cast<uint4*>(stage_ptr + off[it]) = v[it];
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
           if (C == 1) {
-#pragma unroll
-            for (int it = 0; it < TASKS_PER_THREAD; ++it)
-              *reinterpret_cast<uint4*>(a_ring + sa * SK_A_BYTES + off[it]) = v[it];
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(fulla_bar(sa));
+            mbar_arrive(fulla_bar(grp));
           } else {
-            // This CTA's rows of the stage go into every CTA's ring as asynchronous stores that
-            // count their bytes on the destination's fullA barrier; the barrier completes when all
-            // 16 KiB of the stage (from all C CTAs) have landed and the local arrival below is in.
-            if (gtid == 0) mbar_arrive_expect_tx(fulla_bar(sa), SK_A_BYTES);
-#pragma unroll
-            for (int it = 0; it < TASKS_PER_THREAD; ++it)
+            // The stage is complete here once the group's warps have arrived and the other CTAs'
+            // rows have been copied in; the copies count their bytes on this barrier.
+            if (gtid == 0) mbar_arrive_expect_tx(fulla_bar(grp), SK_A_BYTES - PART_BYTES);
+            else mbar_arrive(fulla_bar(grp));
+            // The warp that stores last sends this CTA's rows to the other CTAs with one bulk
+            // copy each.  The counter only grows: a stage is reused after its barrier has
+            // completed, so the counts of two uses never mix.
+            __threadfence_block();
+            const uint32_t n = atomicAdd(&gen_count[grp], 1u);
+            if ((n % GROUP_WARPS) == GROUP_WARPS - 1) {
+              __threadfence_block();
 #pragma unroll
               for (int q = 0; q < C; ++q)
-                st_async_cluster_v4(ring_base[q] + sa * SK_A_BYTES + off[it], v[it], peer_fulla[q] + 8u * sa);
+                if (q != (int)rank)
+                  bulk_copy_to_cluster(peer_part[q], stage_smem + rank * PART_BYTES, PART_BYTES, peer_fulla[q]);
+            }
           }
-          if (++sa == SK_A_STAGES) { sa = 0; pha ^= 1u; }
         }
+        pha ^= 1u;
       }
+      step0 += len;
       ok = ok && mbar_wait_warp(accfull_bar, (uint32_t)seg & 1u, abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();
