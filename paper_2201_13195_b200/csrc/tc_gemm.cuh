@@ -75,6 +75,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+  MBAR_PEEK_DECLARE();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();       // 0 = leader of the pair
   const bool leader = rank == 0;
@@ -163,6 +164,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int s = 0;
       uint32_t ph = 0;
       int it = 0;                               // tiles done by this pair
+      MBAR_PEEK_CLUSTER(0, full_bar(0), 0u);    // every stage's barrier is tested one stage ahead
       for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++it) {
         const int buf = it & 1;
         // the epilogues of both CTAs must have drained this accumulator buffer (two tiles ago)
@@ -171,20 +173,31 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = (mbar_wait_cluster_warp(full_bar(s), ph, abort_flag, p.status));
-          if (!ok) break;
+          uint32_t ready;
+          MBAR_PEEK_RESULT(0, ready);
+          if (!__all_sync(0xffffffffu, ready != 0)) {
+            ok = (mbar_wait_cluster_warp(full_bar(s), ph, abort_flag, p.status));
+            if (!ok) break;
+          }
           tc_fence_after();
           const uint64_t ad = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
           const uint64_t bd = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
-          if (elect_one()) {
+          const int s_next = (s + 1 == STAGES) ? 0 : s + 1;
+          const uint32_t ph_next = (s_next == 0) ? (ph ^ 1u) : ph;
+          const bool issuer = elect_one();
+          if (issuer) {
 #pragma unroll
             for (int j = 0; j < BK / UMMA_K; ++j)
               umma_bf16_pair(d_tmem, ad + j * a_kstep, bd + j * b_kstep, idesc, (kb | j) != 0 ? 1u : 0u);
+          }
+          MBAR_PEEK_CLUSTER(0, full_bar(s_next), ph_next);   // travels while the commits are issued
+          if (issuer) {
             umma_commit_pair(empty_bar(s));
             umma_commit_pair(empty_bar(s) + peer_delta);
           }
           __syncwarp();
-          if (++s == STAGES) { s = 0; ph ^= 1u; }
+          s = s_next;
+          ph = ph_next;
         }
         if (ok) {
           if (elect_one()) {
