@@ -244,8 +244,8 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
                  : C == 2 ? cudaLaunchKernelEx(&cfg, tc::sketch_kernel<2>, tmB, p, pk)
                           : cudaLaunchKernelEx(&cfg, tc::sketch_kernel<1>, tmB, p, pk);
   if (le != cudaSuccess) return RMM_ERR_CUDA;
-  dim3 rgrid((unsigned)(p.sched.tiles() * per_tile), tc::SK_BM);
-  tc::sketch_reduce_kernel<<<rgrid, 128, 0, stream>>>(p, c, reinterpret_cast<__nv_bfloat16*>(out),
+  dim3 rgrid((unsigned)(p.sched.tiles() * per_tile), tc::SK_BN / tc::SKR_CHUNK);
+  tc::sketch_reduce_kernel<<<rgrid, tc::SK_BM, 0, stream>>>(p, c, reinterpret_cast<__nv_bfloat16*>(out),
                                                       reinterpret_cast<__nv_bfloat16*>(ones_out));
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }

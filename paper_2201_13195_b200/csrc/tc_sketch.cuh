@@ -542,7 +542,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
         const int q = warp & 3;                 // tensor-memory lane quarter of this warp
         const int cgroup = gw >> 2;             // 4 warps share a quarter: 128 columns each
         float* slot = p.partial + (sg.slot * C + rank) * (long long)SK_TILE_ELEMS;
-        float* prow = slot + (long long)(q * 32 + lane) * SK_BN;
+        float* prow = slot + (long long)(q * 32 + lane) * 4;   // this lane's row, quad-major layout
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
           const int c = cgroup * 4 + cc;
@@ -551,7 +551,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
           tmem_ld_wait();
 #pragma unroll
           for (int g = 0; g < 8; ++g)
-            *reinterpret_cast<uint4*>(prow + c * 32 + g * 4) = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            *reinterpret_cast<uint4*>(prow + (long long)(c * 8 + g) * SK_BM * 4) = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
         }
       }
       tc_fence_before();
@@ -570,50 +570,56 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
   if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
+// Layout of a partial tile (128 rows x 512 columns, fp32): column quads are outermost, element
+// (r, col) sits at float index ((col / 4) * 128 + r) * 4 + col % 4.  The accumulator comes out
+// of tensor memory one row per lane, so a warp's 16-byte stores of one quad are 512 contiguous
+// bytes, and the reduce kernel, one row per thread, reads them back the same way.
+__host__ __device__ inline long long sketch_partial_index(int r, int col) {
+  return ((long long)(col >> 2) * SK_BM + r) * 4 + (col & 3);
+}
+
 // Adds the partial tiles of each output tile in schedule order, scales, rounds to bf16.
-// grid = (tile groups * C, 128 rows), block = 128 threads: thread t owns columns 4t .. 4t+3 of one
-// row; blockIdx.x = C * tile group + rank of the CTA that produced the 512-column block.
-// All loads of a thread are independent, so the kernel runs at memory speed.
-constexpr int SKR_MAX_SLOTS = 8;     // partial tiles summed per batch of loads
-__global__ void __launch_bounds__(128)
+// grid = (tile groups * C, 16 column chunks), block = 128 threads: thread t owns row t of the
+// tile and the 32 columns of the chunk; blockIdx.x = C * tile group + rank of the CTA that
+// produced the 512-column block.  The loads of a thread are independent of each other.
+constexpr int SKR_CHUNK = 32;        // columns per block of the reduce kernel
+__global__ void __launch_bounds__(SK_BM)
 sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ ones_out) {
   const SketchSchedule& sc = p.sched;
   const int per_tile = sc.cluster;      // partial tiles (CTAs) per schedule tile
   const int tile = blockIdx.x / per_tile, rank = blockIdx.x % per_tile;
   const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
   const long long n0 = ((long long)(tile % sc.tiles_n) * sc.cluster + rank) * SK_BN;
-  const int r = blockIdx.y;
+  const int r = threadIdx.x;
   const long long j = m0 + r;
-  const int col = threadIdx.x * 4;
-  if (j >= p.rows || n0 + col >= p.cols) return;
-  long long slots[SKR_MAX_SLOTS];
-  int ns = 0;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  const long long off = (long long)r * SK_BN + col;
-  auto flush = [&]() {
-    float4 v[SKR_MAX_SLOTS];
+  const int col0 = blockIdx.y * SKR_CHUNK;
+  if (j >= p.rows || n0 + col0 >= p.cols) return;
+  float4 acc[SKR_CHUNK / 4];
 #pragma unroll
-    for (int i = 0; i < SKR_MAX_SLOTS; ++i)
-      if (i < ns) v[i] = __ldcs(reinterpret_cast<const float4*>(p.partial + (slots[i] * per_tile + rank) * (long long)SK_TILE_ELEMS + off));
-#pragma unroll
-    for (int i = 0; i < SKR_MAX_SLOTS; ++i)
-      if (i < ns) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
-    ns = 0;
-  };
+  for (int g = 0; g < SKR_CHUNK / 4; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+  const long long off = sketch_partial_index(r, col0);
   sketch_for_each_slot_of_tile(sc, tile, [&](long long slot_index) {
-    slots[ns++] = slot_index;
-    if (ns == SKR_MAX_SLOTS) flush();
+    const float* src = p.partial + (slot_index * per_tile + rank) * (long long)SK_TILE_ELEMS + off;
+    float4 v[SKR_CHUNK / 4];
+#pragma unroll
+    for (int g = 0; g < SKR_CHUNK / 4; ++g) v[g] = __ldcs(reinterpret_cast<const float4*>(src + (long long)g * SK_BM * 4));
+#pragma unroll
+    for (int g = 0; g < SKR_CHUNK / 4; ++g) { acc[g].x += v[g].x; acc[g].y += v[g].y; acc[g].z += v[g].z; acc[g].w += v[g].w; }
   });
-  flush();
   const bool is_ones = p.ones_row && j == p.b_proj;
   const float s = is_ones ? 1.0f : scale;
-  __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * s, acc.y * s), hi = __floats2bfloat162_rn(acc.z * s, acc.w * s);
-  uint2 o = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-  // cols is a multiple of 8 and col a multiple of 4: the 4 columns are all inside or all outside
-  if (is_ones) {
-    if (ones_out) *reinterpret_cast<uint2*>(ones_out + n0 + col) = o;
-  } else {
-    *reinterpret_cast<uint2*>(out + j * p.cols + n0 + col) = o;
+  __nv_bfloat16* dst = is_ones ? ones_out : out + j * p.cols;
+  if (dst == nullptr) return;
+  dst += n0 + col0;
+  // cols is a multiple of 8: the 8 columns of a 16-byte store are all inside or all outside
+#pragma unroll
+  for (int g = 0; g < SKR_CHUNK / 8; ++g) {
+    if (n0 + col0 + 8 * g >= p.cols) break;
+    const float4 a = acc[2 * g], b = acc[2 * g + 1];
+    __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x * s, a.y * s), h1 = __floats2bfloat162_rn(a.z * s, a.w * s);
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(b.x * s, b.y * s), h3 = __floats2bfloat162_rn(b.z * s, b.w * s);
+    *reinterpret_cast<uint4*>(dst + 8 * g) = make_uint4(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1),
+                                                        *reinterpret_cast<uint32_t*>(&h2), *reinterpret_cast<uint32_t*>(&h3));
   }
 }
 
