@@ -29,7 +29,7 @@ METRIC = "RMM linear fwd+bwd TFLOP/s (bf16)"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "large_ffn_up_rho0.1"
 # (workload, step) -> dram__bytes_read.sum + dram__bytes_write.sum per token row of the kernel's
-# input, from profiles/sketch_kernel_n4096_dout4096_k1638.md: (33.62 MB + 0.74 MB) / 4096 tokens.
+# input, from an ncu capture of sketch_kernel<2> at 4096 tokens: (33.62 MB + 0.74 MB) / 4096.
 NCU_DRAM_BYTES_PER_TOKEN = {("large_ffn_up_rho0.1", "sdy"): (33.622272e6 + 0.74112e6) / 4096}
 
 STEP_ORDER = ("y", "sketch", "dx", "sdy", "dw", "db")
@@ -280,8 +280,8 @@ def main():
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
                 "peak_kind": f"sustained bf16 GEMM, of {peaks['source']}", "frac_of_burst": achieved / peaks["bf16_tflops"],
                 "traffic": None, "algorithmic_flops_per_launch": flops_of[dom]}
-    # DRAM bytes per launch of the dominant step, from the ncu capture summarised under profiles/
-    # (taken at 4096 tokens; the reads are the dY stream and grow in proportion to the tokens).
+    # DRAM bytes per launch of the dominant step, from an ncu capture taken at 4096 tokens; the
+    # reads are the dY stream and grow in proportion to the tokens.
     ncu_traffic = NCU_DRAM_BYTES_PER_TOKEN.get((w.name, dom))
     if ncu_traffic is not None:
         roofline["traffic"] = ncu_traffic * w.n_tokens

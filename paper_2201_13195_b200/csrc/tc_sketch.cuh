@@ -9,13 +9,14 @@
 // memory of an SM (512 fp32 columns) accumulates it, so that every generated entry of S
 // is used 512 times by the CTA that holds it.
 //
-// Sharing S across a cluster.  Generating the normals is plain ALU work (about 29
-// instructions each) and would cost more time than the MMAs that consume them.  CTAs that
-// compute the same sketch rows for neighbouring 512-column blocks therefore form a
-// thread-block cluster of C (1, 2 or 4): each CTA generates 128/C rows of every S^T stage and
-// stores them, with ordinary distributed-shared-memory stores, into the operand ring of
-// all C CTAs, so each generated entry feeds C x 512 columns.  Every CTA runs its own
-// TMA ring for its B columns, its own MMAs and its own accumulator.
+// Sharing S across a cluster.  Generating the normals is plain ALU work (about 24
+// instructions each) and takes about as many issue slots as the MMAs that consume them take
+// tensor cycles.  CTAs that compute the same sketch rows for neighbouring 512-column blocks
+// therefore form a thread-block cluster of C (1 or 2; 4 compiles but too few such clusters are
+// co-resident): each CTA generates 128/C rows of every S^T stage into its own operand ring and
+// sends that block to the other CTAs with one bulk shared-to-shared copy each, counted on the
+// destination's full barrier, so each generated entry feeds C x 512 columns.  Every CTA runs
+// its own TMA ring for its B columns, its own MMAs and its own accumulator.
 //
 // Stream-K.  There are far fewer tiles than SMs and each has a long contraction (all tokens),
 // so (tile group, 64-token step) units are distributed over the clusters by a static
@@ -27,12 +28,13 @@
 // db for free: when ones_row is set, row index B_proj of S^T is a row of ones, so row
 // B_proj of the result is sum_n dY[n][:] (Eq. 3); the reduce kernel stores it, unscaled.
 //
-// Warp roles: warp 0 TMA producer (B), warp 1 tensor-memory owner and MMA issuer, warps
-// 2..17 generate S tiles and drain the accumulator.  A stages hold 64 tokens, B stages 32
-// tokens.  Barriers of a CTA: fullA[s] (C x generating warps: the stage is complete in this
-// CTA's ring), emptyA[s] (C commits: every CTA of the cluster has consumed the stage, so it
-// may be overwritten everywhere), fullB / emptyB (TMA ring), accfull / accempty.  All waits
-// are bounded.
+// Warp roles: warp 0 TMA producer (B); warps 1-2 MMA issuers, one per 256-column half of the
+// accumulator (warp 1 owns the tensor memory); warps 3..18 generate S tiles, in four groups that
+// each own one ring stage, and drain the accumulator.  A stages hold 64 tokens, B stages 32
+// tokens.  Barriers of a CTA: fullA[s] (the group's warps + the bytes copied in by the other
+// CTAs: the stage is complete in this CTA's ring), emptyA[s] (2 C commits: every MMA warp of
+// every CTA of the cluster has consumed the stage, so it may be overwritten everywhere),
+// fullB / emptyB (TMA ring; 2 commits), accfull / accempty.  All waits are bounded.
 #pragma once
 #include "sketch_rng.cuh"
 #include "tc_common.cuh"
