@@ -148,7 +148,7 @@ def run_reference(args, w):
     if rank != 0:
         return
     from oracle import oracle as O
-    total_budget = 90.0
+    total_budget = args.reference_budget_s
     per_step = total_budget / max(1, args.steps + args.warmup)
     n = pick_sample_tokens(w, per_step)
     for _ in range(args.warmup):
@@ -177,6 +177,23 @@ def workload_config(w):
             "l2": f"inputs larger than L2: about {touched / 1e6:.0f} MB of tensors touched per step, no flush"}
 
 
+# ----------------------------------------------------------------------------- N > 1: independent replicas
+def max_over_ranks(ms_local, device):
+    """Job time = the slowest rank's device time (all ranks get it). One process: the value itself."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms_local)
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(flops_per_replica, world, ms_step):
+    """Whole-job TFLOP/s: every rank runs one replica of the layer (weak scaling, no collective on the data path)."""
+    return world * flops_per_replica / (ms_step * 1e-3) / 1e12
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def main():
     ap = argparse.ArgumentParser()
@@ -187,6 +204,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--reference-budget-s", type=float, default=90.0,
+                    help="wall-clock budget of the whole --impl reference run (sizes its token sample)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = R.WORKLOADS[args.workload]
@@ -255,13 +274,10 @@ def main():
     records = P.rmm_profile_read(min(args.steps, 200) * 6)
     P.rmm_profile_enable(0)
 
-    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, torch.device("cuda", local_rank))
     ms_step = ms_total / args.steps
     fl = w.flops()
-    value = world * fl["total"] / (ms_step * 1e-3) / 1e12
+    value = job_value(fl["total"], world, ms_step)
 
     # ---- per-kernel durations and roofline of the dominant kernel
     per_kernel = {}
