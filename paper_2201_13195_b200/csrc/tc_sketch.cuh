@@ -68,8 +68,9 @@ constexpr int SK_MAX_CTAS = 148;                     // CTAs (all clusters toget
 //      block b of tile t goes to CTA b * tiles_rem + t, so all CTAs of a block walk the
 //      same token range in step;
 //   3. the last, narrower block (width `w_last`) is laid out tile after tile and cut
-//      into ranges of `upc` units, which may span several tiles -- unless that would give a
-//      CTA many short segments, in which case the tiles are cut into equal blocks only.
+//      into ranges of `upl` units, which may span several tiles; `upl` < `upc`, because each
+//      extra segment costs a drain of the accumulator -- or, when that is cheaper, the tiles
+//      are cut into equal blocks only (make_sketch_schedule compares the candidates).
 // Every (CTA, tile) intersection is one segment = one fp32 partial tile (slot).
 struct SketchSchedule {
   int cluster;             // C: CTAs per cluster = 512-column blocks per tile group
@@ -80,7 +81,8 @@ struct SketchSchedule {
   int upc;                 // units per CTA in the blocked part
   int full_blocks;         // blocks of width upc
   int w_last;              // width of the last block (0 if none)
-  long long lcm_last;      // lcm(upc, w_last)
+  int upl;                 // units per CTA in the last block's line
+  long long lcm_last;      // lcm(upl, w_last)
 
   __host__ __device__ int tiles() const { return tiles_m * tiles_n; }
   __host__ __device__ long long num_slots() const { return (long long)tiles() + num_ctas; }
@@ -143,8 +145,8 @@ __host__ __device__ inline bool sketch_next_segment(const SketchSchedule& sc, in
   if (sc.w_last == 0) return false;
   const int ci = cta - nfull;
   const long long total = (long long)sc.tiles_rem * sc.w_last;
-  const long long begin = (long long)ci * sc.upc;
-  const long long end = begin + sc.upc < total ? begin + sc.upc : total;
+  const long long begin = (long long)ci * sc.upl;
+  const long long end = begin + sc.upl < total ? begin + sc.upl : total;
   if (it == sc.rounds) { cursor = begin; }
   if (cursor >= end) return false;
   const int t = (int)(cursor / sc.w_last);
@@ -172,10 +174,10 @@ __host__ __device__ inline void sketch_for_each_slot_of_tile(const SketchSchedul
   const int t = tile - base_tile;
   for (int b = 0; b < sc.full_blocks; ++b) f(sc.slot_block(b, t));
   if (sc.w_last > 0) {
-    const int ci_first = (int)(((long long)t * sc.w_last) / sc.upc);
-    const int ci_last = (int)((((long long)t + 1) * sc.w_last - 1) / sc.upc);
+    const int ci_first = (int)(((long long)t * sc.w_last) / sc.upl);
+    const int ci_last = (int)((((long long)t + 1) * sc.w_last - 1) / sc.upl);
     for (int ci = ci_first; ci <= ci_last; ++ci) {
-      const long long cs = (long long)ci * sc.upc, ts = (long long)t * sc.w_last;
+      const long long cs = (long long)ci * sc.upl, ts = (long long)t * sc.w_last;
       f(sc.slot_last(ci, t, cs > ts ? cs : ts));
     }
   }
@@ -200,33 +202,56 @@ inline SketchSchedule make_sketch_schedule(long long rows, long long cols, long 
   s.rounds = tiles / max_ctas;
   s.tiles_rem = tiles % max_ctas;
   s.num_ctas = max_ctas;
-  s.upc = 0; s.full_blocks = 0; s.w_last = 0; s.lcm_last = 1;
+  s.upc = 0; s.full_blocks = 0; s.w_last = 0; s.upl = 1; s.lcm_last = 1;
   if (s.tiles_rem > 0) {
+    // Every segment ends with a drain of the accumulator that the next segment has to wait for:
+    // about kSegCost steps' worth.  CTAs of the last block's line work on several tiles, so they
+    // get fewer units than the CTAs that own a full block.  Candidates: every full-block width
+    // from the even share upwards (the rest of each tile forms the last block, shared by the
+    // CTAs that are left), and equal blocks with no last block; the one whose busiest CTA
+    // finishes first wins.
+    constexpr int kSegCost = 14;
     const long long total = (long long)s.tiles_rem * s.ksteps;
-    s.upc = (int)((total + max_ctas - 1) / max_ctas);
-    if (s.upc < 4 && s.upc < s.ksteps) s.upc = s.ksteps < 4 ? s.ksteps : 4;   // no slivers
-    s.full_blocks = s.ksteps / s.upc;
-    s.w_last = s.ksteps - s.full_blocks * s.upc;
-    if (s.w_last > 0 && s.full_blocks > 0) {
-      // A narrow last block gives a few CTAs many short segments, each of which costs a drain of
-      // the accumulator (about kSegCost steps' worth).  Compare with cutting every tile into
-      // full_blocks equal blocks instead (fewer CTAs busy, one segment each) and take the
-      // schedule whose busiest CTA finishes first.
-      constexpr int kSegCost = 8;
-      const int segs_last = (s.upc + s.w_last - 1) / s.w_last + 1;
-      const int cost_stream = s.upc + kSegCost * segs_last;
-      const int upc_even = (s.ksteps + s.full_blocks - 1) / s.full_blocks;
-      const int cost_even = upc_even + kSegCost;
-      if (cost_even <= cost_stream) {
-        s.upc = upc_even;
-        s.full_blocks = (s.ksteps + s.upc - 1) / s.upc;
-        s.w_last = 0;
+    int upc0 = (int)((total + max_ctas - 1) / max_ctas);
+    if (upc0 < 4 && upc0 < s.ksteps) upc0 = s.ksteps < 4 ? s.ksteps : 4;   // no slivers
+    long long best_cost = -1;
+    for (int u1 = upc0; u1 <= s.ksteps; ++u1) {
+      const int fb = s.ksteps / u1;
+      const int wl = s.ksteps - fb * u1;
+      const long long left = (long long)max_ctas - (long long)fb * s.tiles_rem;   // CTAs for the last line
+      long long cost;
+      int u2 = 1;
+      if (wl == 0) {
+        if (left < 0) continue;
+        cost = u1 + kSegCost;
+      } else {
+        if (left < 1) continue;
+        u2 = (int)(((long long)s.tiles_rem * wl + left - 1) / left);
+        const int segs = (u2 + wl - 1) / wl + 1;
+        const long long c2 = u2 + (long long)kSegCost * segs;
+        cost = u1 + kSegCost > c2 ? u1 + kSegCost : c2;
+      }
+      if (best_cost < 0 || cost < best_cost) {
+        best_cost = cost;
+        s.upc = u1; s.full_blocks = fb; s.w_last = wl; s.upl = u2;
       }
     }
-    if (s.w_last > 0) s.lcm_last = (long long)s.upc / gcd_ll(s.upc, s.w_last) * s.w_last;
-    const long long last_ctas = s.w_last > 0 ? ((long long)s.tiles_rem * s.w_last + s.upc - 1) / s.upc : 0;
+    {   // equal blocks: every tile cut into nb blocks of the same width, one segment per CTA
+      const int nb_max = max_ctas / s.tiles_rem;
+      for (int nb = 1; nb <= nb_max && nb <= s.ksteps; ++nb) {
+        const int ue = (s.ksteps + nb - 1) / nb;
+        if (ue < 4 && ue < s.ksteps) break;
+        const long long cost = ue + kSegCost;
+        if (best_cost < 0 || cost <= best_cost) {
+          best_cost = cost;
+          s.upc = ue; s.full_blocks = (s.ksteps + ue - 1) / ue; s.w_last = 0; s.upl = 1;
+        }
+      }
+    }
+    if (s.w_last > 0) s.lcm_last = (long long)s.upl / gcd_ll(s.upl, s.w_last) * s.w_last;
+    const long long last_ctas = s.w_last > 0 ? ((long long)s.tiles_rem * s.w_last + s.upl - 1) / s.upl : 0;
     const long long used = (long long)s.full_blocks * s.tiles_rem + last_ctas;
-    if (s.rounds == 0) s.num_ctas = (int)used;          // never more than max_ctas by construction of upc
+    if (s.rounds == 0) s.num_ctas = (int)used;          // never more than max_ctas by construction
   }
   return s;
 }
