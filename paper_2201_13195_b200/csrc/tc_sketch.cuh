@@ -29,12 +29,13 @@
 // B_proj of the result is sum_n dY[n][:] (Eq. 3); the reduce kernel stores it, unscaled.
 //
 // Warp roles: warp 0 TMA producer (B); warps 1-2 MMA issuers, one per 256-column half of the
-// accumulator (warp 1 owns the tensor memory); warps 3..18 generate S tiles, in four groups that
-// each own one ring stage, and drain the accumulator.  A stages hold 64 tokens, B stages 32
-// tokens.  Barriers of a CTA: fullA[s] (the group's warps + the bytes copied in by the other
-// CTAs: the stage is complete in this CTA's ring), emptyA[s] (2 C commits: every MMA warp of
-// every CTA of the cluster has consumed the stage, so it may be overwritten everywhere),
-// fullB / emptyB (TMA ring; 2 commits), accfull / accempty.  All waits are bounded.
+// accumulator (warp 1 owns the tensor memory); warps 3..14 generate S tiles, in three groups of
+// four that each own one ring stage, and drain the accumulator.  A ring: 3 stages of 64 tokens;
+// B ring: 5 stages of 32 tokens (the B ring is the latency-critical one: it holds 2.5 K-steps).
+// Barriers of a CTA: fullA[s] (the group's warps + the bytes copied in by the other CTAs: the
+// stage is complete in this CTA's ring), emptyA[s] (2 C commits: every MMA warp of every CTA of
+// the cluster has consumed the stage, so it may be overwritten everywhere), fullB / emptyB (TMA
+// ring; 2 commits), accfull / accempty.  All waits are bounded.
 #pragma once
 #include "sketch_rng.cuh"
 #include "tc_common.cuh"
@@ -43,12 +44,15 @@ namespace rmm {
 namespace tc {
 
 constexpr int SK_BM = 128, SK_BN = 512, SK_AK = 64, SK_BK = 32;
-constexpr int SK_A_STAGES = 4, SK_B_STAGES = 4;
+constexpr int SK_A_STAGES = 3, SK_B_STAGES = 5;
 constexpr int SK_A_BYTES = SK_BM * SK_AK * 2;        // 16 KiB
 constexpr int SK_B_BYTES = SK_BN * SK_BK * 2;        // 32 KiB
 constexpr int SK_B_SLAB = 64 * SK_BK * 2;            // [32 tokens][64 columns] = 4 KiB
 constexpr int SK_STAGGER = 2;                        // steps by which neighbouring tile rows are offset
-constexpr int SK_GEN_WARPS = 16;
+constexpr int SK_GEN_GROUPS = SK_A_STAGES;  // one generator warp group per ring stage: group g fills stage g.
+// (A stage must have one producer group: barrier waits only see the parity of a phase, and two
+// groups taking turns on one stage could get two phases apart.)
+constexpr int SK_GEN_WARPS = 4 * SK_GEN_GROUPS;
 constexpr int SK_GEN_THREADS = 32 * SK_GEN_WARPS;
 constexpr int SK_MMA_WARPS = 2;            // each issues the MMAs of one 256-column half of the tile
 constexpr int SK_THREADS = 32 * (1 + SK_MMA_WARPS) + SK_GEN_THREADS;
@@ -322,14 +326,15 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
   uint32_t* gen_count = tmem_slot + 2;           // generator warps that have stored their part of a stage
 
   // tasks = (row, 16-byte chunk) pairs of a stage; this CTA generates rows [rank*128/C, (rank+1)*128/C).
-  // The generator warps form one group per ring stage: group g fills stage g of the ring, i.e.
-  // the K-steps g, g + 4, ... of this CTA's sequence.  The groups run out of phase, so the stores,
-  // fences and barrier round trips of one group are covered by the arithmetic of the others.
+  // The generator warps form one group per ring stage: group g produces the K-steps g,
+  // g + SK_A_STAGES, ... of this CTA's sequence, all of which go into ring stage g.  The groups
+  // run out of phase, so the stores, fences and barrier round trips of one are covered by the
+  // arithmetic of the others.
   constexpr int TASKS = SK_BM * 8 / C;                                         // per CTA and stage
-  constexpr int GROUP_WARPS = SK_GEN_WARPS / SK_A_STAGES;
+  constexpr int GROUP_WARPS = SK_GEN_WARPS / SK_GEN_GROUPS;
   constexpr int GROUP_THREADS = 32 * GROUP_WARPS;
   constexpr int TASKS_PER_THREAD = TASKS / GROUP_THREADS;
-  static_assert(SK_GEN_WARPS % SK_A_STAGES == 0 && TASKS % GROUP_THREADS == 0, "generator groups");
+  static_assert(SK_GEN_WARPS % SK_GEN_GROUPS == 0 && TASKS % GROUP_THREADS == 0, "generator groups");
 
   MBAR_PEEK_DECLARE();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -491,21 +496,19 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
   } else {
     // ------------------------------------------------------------ S generators + accumulator drain
     const int gw = warp - 1 - SK_MMA_WARPS;
-    const int grp = gw / GROUP_WARPS;            // ring stage that this warp's group fills
+    const int grp = gw / GROUP_WARPS;            // this warp's group
     const int gtid = (gw % GROUP_WARPS) * 32 + lane;   // thread index within the group
     constexpr uint32_t PART_BYTES = SK_A_BYTES / C;   // this CTA's rows of a stage: one contiguous block
-    const uint32_t stage_smem = smem_u32(a_ring) + grp * SK_A_BYTES;
-    uint8_t* const stage_ptr = a_ring + grp * SK_A_BYTES;
-    uint32_t peer_part[C];                       // where that block goes in stage grp of every CTA of the cluster
-    uint32_t peer_fulla[C];                      // fullA[grp] of every CTA of the cluster
+    const uint32_t part_smem = smem_u32(a_ring) + rank * PART_BYTES;   // that block in stage 0 of this CTA's ring
+    uint32_t peer_part[C];                       // the same place in the ring of every CTA of the cluster
+    uint32_t peer_fulla[C];                      // fullA[0] of every CTA of the cluster
     if (C > 1) {
 #pragma unroll
       for (int r = 0; r < C; ++r) {
-        peer_part[r] = mapa_shared(stage_smem + rank * PART_BYTES, r);
-        peer_fulla[r] = mapa_shared(fulla_bar(grp), r);
+        peer_part[r] = mapa_shared(part_smem, r);
+        peer_fulla[r] = mapa_shared(fulla_bar(0), r);
       }
     }
-    uint32_t pha = 0;                            // parity of the group's stage
     int step0 = 0;                               // position of the segment's first K-step in this CTA's sequence
     int seg = 0;
     bool ok = true;
@@ -516,9 +519,12 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       const int tile = sg.tile;
       const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
       const int len = sg.ks1 - sg.ks0;
-      // the group's first step of this segment: the first i with (step0 + i) % stages == grp
-      for (int i = (grp - step0) & (SK_A_STAGES - 1); i < len; i += SK_A_STAGES) {
+      // the group's first step of this segment: the first i with (step0 + i) % groups == grp
+      for (int i = (grp + SK_GEN_GROUPS - step0 % SK_GEN_GROUPS) % SK_GEN_GROUPS; i < len; i += SK_GEN_GROUPS) {
         const int ks = sketch_step(sg.ks0, sg.ks1, tile / sc.tiles_n, i);
+        const int step = step0 + i;
+        const int sa = grp;                                         // ring stage of this step (step % stages)
+        const uint32_t pha = (uint32_t)(step / SK_A_STAGES) & 1u;   // and its parity
         // Generate first, into registers: the entries do not depend on the ring, so the wait for
         // the free stage only covers the stores.
         uint4 v[TASKS_PER_THREAD];
@@ -530,36 +536,37 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
           v[it] = sketch_chunk(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
           off[it] = (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
         }
-        const bool freed = (C == 1) ? mbar_wait_warp(emptya_bar(grp), pha ^ 1u, abort_flag, p.status)
-                                    : mbar_wait_cluster_warp(emptya_bar(grp), pha ^ 1u, abort_flag, p.status);
+        const bool freed = (C == 1) ? mbar_wait_warp(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)
+                                    : mbar_wait_cluster_warp(emptya_bar(sa), pha ^ 1u, abort_flag, p.status);
         if (!freed) { ok = false; break; }
+        uint8_t* const stage_ptr = a_ring + sa * SK_A_BYTES;
 #pragma unroll
         for (int it = 0; it < TASKS_PER_THREAD; ++it) *reinterpret_cast<uint4*>(stage_ptr + off[it]) = v[it];
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
           if (C == 1) {
-            mbar_arrive(fulla_bar(grp));
+            mbar_arrive(fulla_bar(sa));
           } else {
             // The stage is complete here once the group's warps have arrived and the other CTAs'
             // rows have been copied in; the copies count their bytes on this barrier.
-            if (gtid == 0) mbar_arrive_expect_tx(fulla_bar(grp), SK_A_BYTES - PART_BYTES);
-            else mbar_arrive(fulla_bar(grp));
+            if (gtid == 0) mbar_arrive_expect_tx(fulla_bar(sa), SK_A_BYTES - PART_BYTES);
+            else mbar_arrive(fulla_bar(sa));
             // The warp that stores last sends this CTA's rows to the other CTAs with one bulk
             // copy each.  The counter only grows: a stage is reused after its barrier has
             // completed, so the counts of two uses never mix.
             __threadfence_block();
-            const uint32_t n = atomicAdd(&gen_count[grp], 1u);
+            const uint32_t n = atomicAdd(&gen_count[sa], 1u);
             if ((n % GROUP_WARPS) == GROUP_WARPS - 1) {
               __threadfence_block();
 #pragma unroll
               for (int q = 0; q < C; ++q)
                 if (q != (int)rank)
-                  bulk_copy_to_cluster(peer_part[q], stage_smem + rank * PART_BYTES, PART_BYTES, peer_fulla[q]);
+                  bulk_copy_to_cluster(peer_part[q] + sa * SK_A_BYTES, part_smem + sa * SK_A_BYTES, PART_BYTES,
+                                       peer_fulla[q] + 8u * sa);
             }
           }
         }
-        pha ^= 1u;
       }
       step0 += len;
       ok = ok && mbar_wait_warp(accfull_bar, (uint32_t)seg & 1u, abort_flag, p.status);
@@ -567,12 +574,11 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       tc_fence_after();
       {
         const int q = warp & 3;                 // tensor-memory lane quarter of this warp
-        const int cgroup = gw >> 2;             // 4 warps share a quarter: 128 columns each
+        const int cgroup = gw >> 2;             // index among the SK_GEN_WARPS / 4 warps that share the quarter
         float* slot = p.partial + (sg.slot * C + rank) * (long long)SK_TILE_ELEMS;
         float* prow = slot + (long long)(q * 32 + lane) * 4;   // this lane's row, quad-major layout
 #pragma unroll 1
-        for (int cc = 0; cc < 4; ++cc) {
-          const int c = cgroup * 4 + cc;
+        for (int c = cgroup; c < SK_BN / 32; c += SK_GEN_WARPS / 4) {   // 32-column chunks, dealt round-robin
           uint32_t v[32];
           tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
           tmem_ld_wait();
