@@ -8,7 +8,12 @@ no non-CUDA path: using the package without a built library raises ImportError.
 import importlib
 
 
+_SUBMODULES = ("build", "binding", "run_case")
+
+
 def __getattr__(name):
+    if name in _SUBMODULES:          # `from package import build` must work before the library exists
+        return importlib.import_module("." + name, __name__)
     binding = importlib.import_module(".binding", __name__)
     try:
         return getattr(binding, name)
