@@ -28,9 +28,11 @@ import rmm_inputs as R  # noqa: E402
 METRIC = "RMM linear fwd+bwd TFLOP/s (bf16)"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "large_ffn_up_rho0.1"
-# (workload, step) -> dram__bytes_read.sum + dram__bytes_write.sum per token row of the kernel's
-# input, from an ncu capture of sketch_kernel<2> at 4096 tokens: (33.62 MB + 0.74 MB) / 4096.
-NCU_DRAM_BYTES_PER_TOKEN = {("large_ffn_up_rho0.1", "sdy"): (33.622272e6 + 0.74112e6) / 4096}
+# (workload, step) -> (dram__bytes_read.sum per token row of the kernel's input, dram__bytes_write.sum
+# per launch), from an ncu capture of sketch_kernel<2> at 4096 tokens: 34.30 MB read (the dY stream, in
+# proportion to the tokens), 14.88 MB written (fp32 partial tiles that leave L2; their number follows
+# the schedule, not the token count).
+NCU_DRAM_BYTES = {("large_ffn_up_rho0.1", "sdy"): (34.299136e6 / 4096, 14.875904e6)}
 
 STEP_ORDER = ("y", "sketch", "dx", "sdy", "dw", "db")
 
@@ -298,10 +300,11 @@ def main():
                 "traffic": None, "algorithmic_flops_per_launch": flops_of[dom]}
     # DRAM bytes per launch of the dominant step, from an ncu capture taken at 4096 tokens; the
     # reads are the dY stream and grow in proportion to the tokens.
-    ncu_traffic = NCU_DRAM_BYTES_PER_TOKEN.get((w.name, dom))
+    ncu_traffic = NCU_DRAM_BYTES.get((w.name, dom))
     if ncu_traffic is not None:
-        roofline["traffic"] = ncu_traffic * w.n_tokens
-        roofline["traffic_note"] = "dram read+write of sketch_kernel<2>, ncu at 4096 tokens scaled by tokens"
+        roofline["traffic"] = ncu_traffic[0] * w.n_tokens + ncu_traffic[1]
+        roofline["traffic_note"] = ("dram read+write of sketch_kernel<2>: ncu at 4096 tokens, reads scaled by tokens, "
+                                    "writes (partial tiles) as captured")
 
     # ---- end to end through the host-buffer entry points (pinned host memory)
     e2e = None
