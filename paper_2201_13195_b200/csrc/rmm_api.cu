@@ -182,8 +182,8 @@ struct ScopedTiming {
 template <int AMODE, int BMODE>
 rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, int64_t M, int64_t N, int64_t K,
                      float alpha, int* status, cudaStream_t stream) {
-  CUtensorMap tmA, tmB;
-  bool ok = true;
+  CUtensorMap tmA, tmB, tmC;
+  bool ok = make_tmap(&tmC, c, M, N, 32);        // store boxes of the epilogue: [32 rows][64 columns]
   if (AMODE == tc::A_K) ok &= make_tmap(&tmA, a, M, K, tc::BM);
   if (AMODE == tc::A_MN) ok &= make_tmap(&tmA, a, K, M, tc::BK);
   if (BMODE == tc::B_K) ok &= make_tmap(&tmB, b, N, K, tc::BN_HALF);
@@ -204,7 +204,7 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, tc::gemm_kernel<AMODE, BMODE>, tmA, tmB, p) != cudaSuccess) return RMM_ERR_CUDA;
+  if (cudaLaunchKernelEx(&cfg, tc::gemm_kernel<AMODE, BMODE>, tmA, tmB, tmC, p) != cudaSuccess) return RMM_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
 

@@ -17,6 +17,13 @@
 // the B bytes an SM pulls from L2 and pushes through its shared memory, which is what limits a
 // one-CTA 128 x 256 tile, and it makes room for six pipeline stages instead of four.
 //
+// Epilogue.  Each epilogue warp owns 32 rows of the accumulator.  Per 64 output columns it reads
+// them out of tensor memory, applies alpha and the bias, rounds to bf16, writes a [32 rows][128 B]
+// box into shared memory (128-byte swizzle) and hands it to a TMA store; two boxes per warp, so
+// the conversion of one overlaps the store of the other.  The stores reach L2 as whole 128-byte
+// lines (per-lane 16-byte stores of row fragments cost the Y GEMM a quarter of its time), and
+// the tensor map clips rows and columns beyond the matrix.
+//
 // Warp roles per CTA: warp 0 = TMA producer (its halves), warp 1 = tensor-memory owner and, in
 // the leader CTA (even rank), MMA issuer; warps 2..5 = epilogue.  Barriers: full (leader; TMA
 // bytes of both CTAs landed), empty (both; tcgen05.commit from the leader: the MMAs that read
@@ -39,7 +46,11 @@ constexpr int B_BYTES = BN_HALF * BK * 2;     // 16 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SLAB_BYTES = 64 * BK * 2;       // one [64 k][64 mn] MN-major slab, 8 KiB
 constexpr int TMEM_COLS = 512;                // two 128 x 256 fp32 accumulators per CTA
-constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int NEPI = 4;                       // epilogue warps: one per tensor-memory lane quarter
+constexpr int EPI_COLS = 64;                  // output columns per store box: 128 bytes of bf16
+constexpr int EPI_BOX_BYTES = 32 * EPI_COLS * 2;   // [32 rows][64 columns] = 4 KiB
+constexpr int EPI_BYTES = NEPI * 2 * EPI_BOX_BYTES;   // two boxes per epilogue warp
+constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 enum : int { A_K = 0, A_MN = 1 };
 enum : int { B_K = 0, B_MN = 1 };
@@ -58,15 +69,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-constexpr int NEPI = 4;   // epilogue warps: one per tensor-memory lane quarter
-
 template <int AMODE, int BMODE>
 __global__ void __launch_bounds__(64 + 32 * NEPI, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmC, GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES + EPI_BYTES);
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
@@ -214,7 +224,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int q = warp & 3;                       // tensor-memory lane quarter this warp may read
     const __nv_bfloat16* bias = reinterpret_cast<const __nv_bfloat16*>(p.bias);
     const uint32_t accempty_leader0 = mapa_shared(accempty_bar(0), 0);
+    const uint32_t box0 = sbase + STAGES * STAGE_BYTES + (uint32_t)(warp - 2) * 2 * EPI_BOX_BYTES;   // this warp's two boxes
+    const uint32_t row_off = (uint32_t)lane * 128u, sw = (uint32_t)(lane & 7);
+    if (lane == 0) tma_prefetch_desc(&tmC);
     int it = 0;
+    uint32_t nbox = 0;                            // boxes filled so far: box nbox & 1 is next
     for (int tile = pair; tile < num_tiles; tile += num_pairs, ++it) {
       const int buf = it & 1;
       const bool acc_ready =
@@ -222,45 +236,55 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if (!acc_ready) break;
       tc_fence_after();
       const int64_t m0 = (int64_t)(tile / tiles_n) * PAIR_M + (int64_t)rank * BM, n0 = (int64_t)(tile % tiles_n) * BN;
-      const int64_t row = m0 + q * 32 + lane;
-      __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc;
+      const int64_t row0 = m0 + q * 32;           // first row of this warp's boxes
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c * 32), v);
-        tmem_ld_wait();
-        if (row < p.M) {
+      for (int cb = 0; cb < BN / EPI_COLS; ++cb, ++nbox) {
+        const uint32_t box = box0 + (nbox & 1u) * EPI_BOX_BYTES;
+        // the store that read this box two boxes ago must have finished reading it
+        if (lane == 0) bulk_wait_group_read<1>();
+        __syncwarp();
+#pragma unroll
+        for (int h = 0; h < EPI_COLS / 32; ++h) {
+          uint32_t v[32];
+          tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + cb * EPI_COLS + h * 32), v);
+          tmem_ld_wait();
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
-            const int64_t col = n0 + c * 32 + g * 8;
-            if (col < p.N) {
-              float f[8];
+            const int64_t col = n0 + cb * EPI_COLS + h * 32 + g * 8;
+            float f[8];
 #pragma unroll
-              for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[g * 8 + i]) * p.alpha;
-              if (bias) {
-                const uint4 bv = *reinterpret_cast<const uint4*>(bias + col);
-                const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
+            for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[g * 8 + i]) * p.alpha;
+            if (bias && col < p.N) {              // N is a multiple of 8: a group of 8 columns is all in or all out
+              const uint4 bv = *reinterpret_cast<const uint4*>(bias + col);
+              const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  f[2 * i] += __uint_as_float(bw[i] << 16);
-                  f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
-                }
+              for (int i = 0; i < 4; ++i) {
+                f[2 * i] += __uint_as_float(bw[i] << 16);
+                f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
               }
-              uint4 o;
-              o.x = pack_bf16x2(f[0], f[1]);
-              o.y = pack_bf16x2(f[2], f[3]);
-              o.z = pack_bf16x2(f[4], f[5]);
-              o.w = pack_bf16x2(f[6], f[7]);
-              *reinterpret_cast<uint4*>(crow + col) = o;
             }
+            // row `lane` of the box, 16-byte chunk 4h + g, at its swizzled position
+            const uint32_t dst = box + row_off + ((((uint32_t)(4 * h + g)) ^ sw) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16x2(f[0], f[1])),
+                         "r"(pack_bf16x2(f[2], f[3])), "r"(pack_bf16x2(f[4], f[5])), "r"(pack_bf16x2(f[6], f[7]))
+                         : "memory");
           }
         }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          const int64_t col0 = n0 + cb * EPI_COLS;
+          if (row0 < p.M && col0 < p.N) tma_store_2d(&tmC, box, (int)col0, (int)row0);
+          bulk_commit_group();
+        }
       }
-      // hand the buffer back to the MMA issuer in the leader CTA
+      // every read of the accumulator buffer is done: hand it back to the MMA issuer in the leader CTA
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(accempty_leader0 + 8u * buf);
     }
+    if (lane == 0) bulk_wait_group_all();         // the boxes must outlive their stores
+    __syncwarp();
   }
   // ---------------------------------------------------------------- teardown
   if (*abort_flag) {
