@@ -142,3 +142,11 @@ def test_sketch_schedule_covers_every_unit_once(rows, cols, tokens, ctas):
     # no CTA is left with a long tail of tiny segments
     nseg = collections.Counter(c for c, _, ks0, ks1, _ in segs if ks1 - ks0 < ksteps)
     assert not nseg or max(nseg.values()) <= 6
+
+
+def test_rmm_linear_bproj_rule_matches_harness_rule():
+    """The module's B_proj = round(rho * tokens) is the rule the workloads use."""
+    import rmm_inputs as R
+    from paper_2201_13195_b200.rmm_linear import bproj_from_rho
+    for n, rho in ((4096, 0.1), (4096, 0.2), (4096, 0.5), (4096, 0.9), (16384, 0.1), (512, 0.5), (7, 0.01), (3, 1.0)):
+        assert bproj_from_rho(n, rho) == R.bproj_from_rho(n, rho) >= 1
