@@ -196,6 +196,37 @@ rmm_status rmm_bias_grad_static(const void* dY, int64_t N, int64_t D_out, rmm_dt
                                 void* cuda_stream);
 
 /*
+ * Variance diagnostics of the randomized weight gradient (Section 2.3).  For one layer's
+ * actual X [N, D_in] and dY [N, D_out] (the paper's X and Y of Lemmas 1 and 2) it computes
+ *   out[0] = |X|_F^2            out[1] = |dY|_F^2
+ *   out[2] = sum_n |x_n|^2 |dy_n|^2
+ *   out[3] = |X^T dY|_F^2       (the squared norm of the exact gradient, Eq. 3)
+ *   out[4] = D^2_SGD = N/(N-1) out[2] - out[3]/(N-1)                        (Lemma 1, Eq. 9)
+ *   out[5] = D^2_RMM = E |X^T S S^T dY - X^T dY|_F^2 for the given sketch with the fourth
+ *            moment of its entries kept: (out[0] out[1] + out[3]) / B_proj for Gaussian S,
+ *            (out[0] out[1] + out[3] - 2 out[2]) / B_proj for Rademacher S, 0 for S = I
+ *   out[6] = (out[0] out[1] - out[3]) / B_proj, the expression Lemma 2, Eq. 11 prints
+ *            (it drops the fourth moment; it equals out[5] only when X^T dY = 0)
+ *   out[7] = alpha = out[3] / (out[0] out[1])                               (Theorem 1, Eq. 13)
+ * It needs X, so it is a debugging aid for a probed layer, not part of a training step that
+ * wants the memory saving (the paper, too, probes single layers: Section 4.2).
+ *   in : X, dY (device, bf16 only: RMM_ERR_UNSUPPORTED for RMM_DTYPE_F32), N >= 2,
+ *        1 <= B_proj <= N, dist as in rmm_forward
+ *   out: out = 8 doubles in DEVICE memory (16-byte aligned), written on the stream;
+ *        dW_exact (nullable) = the exact gradient dY^T X [D_out, D_in] in bf16, which the
+ *        probe computes on the way
+ *   workspace: at least rmm_variance_probe_workspace_bytes(N, D_in, D_out) bytes, 256-byte
+ *        aligned, caller-owned; it also receives the device status word that
+ *        rmm_last_device_status() reads.
+ * Sums are accumulated in fp32 inside a row or a tensor-core tile and in fp64 across them,
+ * in a fixed order (the result is reproducible).
+ */
+size_t rmm_variance_probe_workspace_bytes(int64_t N, int64_t D_in, int64_t D_out);
+rmm_status rmm_variance_probe(const void* X, const void* dY, int64_t N, int64_t D_in, int64_t D_out,
+                              int64_t B_proj, rmm_dist dist, rmm_dtype dt, double* out, void* dW_exact,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Host-buffer convenience wrappers (end-to-end path): the tensor arguments are HOST
  * pointers (pinned memory recommended); the device buffers dev_* and the workspace
  * are caller-owned DEVICE scratch of at least the tensors' sizes.  Each call copies

@@ -19,7 +19,8 @@ RMM_DTYPE_BF16, RMM_DTYPE_F32 = 0, 1
 EXPORTS = ("rmm_workspace_bytes", "rmm_forward", "rmm_backward", "rmm_debug_generate_s",
            "rmm_last_device_status", "rmm_status_string", "rmm_host_staging_bytes",
            "rmm_forward_host", "rmm_backward_host", "rmm_profile_enable", "rmm_profile_read",
-           "rmm_bias_grad_static", "rmm_debug_gauss_words", "rmm_debug_sketch_schedule")
+           "rmm_bias_grad_static", "rmm_debug_gauss_words", "rmm_debug_sketch_schedule",
+           "rmm_variance_probe_workspace_bytes", "rmm_variance_probe")
 RMM_BIAS_GRAD_STATIC_MAX_D_OUT = 4096
 STEP_NAMES = ("y", "sketch", "dx", "sdy", "dw", "db")
 
@@ -53,6 +54,10 @@ _lib.rmm_debug_gauss_words.argtypes = [_vp, _i64, _vp, _vp]
 _lib.rmm_debug_gauss_words.restype = _int
 _lib.rmm_debug_sketch_schedule.argtypes = [_i64, _i64, _i64, _int, _int, _vp, _i64, _vp]
 _lib.rmm_debug_sketch_schedule.restype = _i64
+_lib.rmm_variance_probe_workspace_bytes.argtypes = [_i64, _i64, _i64]
+_lib.rmm_variance_probe_workspace_bytes.restype = _sz
+_lib.rmm_variance_probe.argtypes = [_vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _vp, _vp, _vp, _sz, _vp]
+_lib.rmm_variance_probe.restype = _int
 _lib.rmm_profile_enable.argtypes = [_int]
 _lib.rmm_profile_enable.restype = _int
 _lib.rmm_profile_read.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_float), _int]
@@ -176,6 +181,29 @@ def rmm_backward_host(dY, W, X_proj, seed, dist, dX, dW, db, dev_in, dev_out, wo
                                   _ptr(dX), _ptr(dW), _ptr(db), _ptr(dev_in), _ptr(dev_out), _ptr(workspace),
                                   workspace.numel(), _stream_ptr(stream)), "rmm_backward_host")
     return dX, dW, db
+
+
+VARIANCE_FIELDS = ("x_frob2", "dy_frob2", "rownorm_products", "xtdy_frob2", "d2_sgd", "d2_rmm", "d2_rmm_printed", "alpha")
+
+
+def rmm_variance_probe_workspace_bytes(N, D_in, D_out) -> int:
+    return int(_lib.rmm_variance_probe_workspace_bytes(N, D_in, D_out))
+
+
+def rmm_variance_probe(X, dY, B_proj, dist, out=None, dW_exact=None, workspace=None, stream=None):
+    """Device tensor of 8 doubles (VARIANCE_FIELDS) for one layer's X [N, D_in] and dY [N, D_out] (bf16)."""
+    N, D_in = X.shape
+    D_out = dY.shape[1]
+    assert X.is_cuda and dY.is_cuda and X.is_contiguous() and dY.is_contiguous() and dY.shape[0] == N
+    if out is None:
+        out = torch.empty(8, dtype=torch.float64, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(rmm_variance_probe_workspace_bytes(N, D_in, D_out), dtype=torch.uint8,
+                                device=X.device)
+    _check(_lib.rmm_variance_probe(_ptr(X), _ptr(dY), N, D_in, D_out, B_proj, dist, _dtype_code(X), _ptr(out),
+                                   _ptr(dW_exact), _ptr(workspace), workspace.numel(), _stream_ptr(stream)),
+           "rmm_variance_probe")
+    return out
 
 
 def rmm_profile_enable(capacity: int) -> None:

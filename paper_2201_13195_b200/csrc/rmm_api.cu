@@ -13,6 +13,7 @@
 #include "sketch_rng.cuh"
 #include "tc_gemm.cuh"
 #include "tc_sketch.cuh"
+#include "variance_kernels.cuh"
 
 namespace {
 
@@ -179,9 +180,16 @@ struct ScopedTiming {
 // One contraction on the tensor cores.  a/b are row-major bf16 matrices:
 //   A_K : a is [M][K]   A_MN: a is [K][M]
 //   B_K : b is [N][K]   B_MN: b is [K][N]
+// Number of CTAs launch_tc uses for an M x N result (the size of the optional sumsq array is NEPI times this).
+int tc_grid_ctas(int64_t M, int64_t N) {
+  const int64_t tiles = ((N + tc::BN - 1) / tc::BN) * ((M + tc::PAIR_M - 1) / tc::PAIR_M);
+  const int max_pairs = device_state().gemm_pairs;
+  return 2 * (int)(tiles < max_pairs ? tiles : max_pairs);
+}
+
 template <int AMODE, int BMODE>
 rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, int64_t M, int64_t N, int64_t K,
-                     float alpha, int* status, cudaStream_t stream) {
+                     float alpha, int* status, cudaStream_t stream, double* sumsq = nullptr) {
   CUtensorMap tmA, tmB, tmC;
   bool ok = make_tmap(&tmC, c, M, N, 32);        // store boxes of the epilogue: [32 rows][64 columns]
   if (AMODE == tc::A_K) ok &= make_tmap(&tmA, a, M, K, tc::BM);
@@ -191,7 +199,7 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   if (!ok) return RMM_ERR_CUDA;
   tc::GemmParams p;
   p.M = M; p.N = N; p.K = K;
-  p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.status = status;
+  p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.status = status; p.sumsq = sumsq;
   const int64_t tiles = ((N + tc::BN - 1) / tc::BN) * ((M + tc::PAIR_M - 1) / tc::PAIR_M);
   const int max_pairs = device_state().gemm_pairs;
   cudaLaunchConfig_t cfg = {};
@@ -499,6 +507,64 @@ const char* rmm_status_string(rmm_status s) {
     case RMM_ERR_TIMEOUT: return "RMM_ERR_TIMEOUT";
   }
   return "RMM_ERR_UNKNOWN";
+}
+
+// ------------------------------------------------------------------ variance diagnostics
+namespace {
+struct ProbeWorkspace {
+  size_t status_off, row_off, gemm_off, dw_off, total;
+  int row_blocks;
+};
+ProbeWorkspace probe_layout(int64_t N, int64_t D_in, int64_t D_out) {
+  ProbeWorkspace w;
+  const int64_t want = (N + VAR_WARPS - 1) / VAR_WARPS;  // at least one row per warp
+  const int64_t cap = (int64_t)(device_state().num_sms > 0 ? device_state().num_sms : 148) * VAR_BLOCKS_PER_SM;
+  w.row_blocks = (int)(want < cap ? want : cap);
+  if (w.row_blocks > 4096) w.row_blocks = 4096;
+  w.status_off = 0;
+  w.row_off = kAlign;
+  w.gemm_off = w.row_off + align_up((size_t)4096 * 3 * sizeof(double));   // room for any grid of row_norms_kernel
+  w.dw_off = w.gemm_off + align_up((size_t)tc::SK_MAX_CTAS * tc::NEPI * sizeof(double));
+  w.total = w.dw_off + align_up((size_t)D_out * (size_t)D_in * 2);
+  return w;
+}
+}  // namespace
+
+size_t rmm_variance_probe_workspace_bytes(int64_t N, int64_t D_in, int64_t D_out) {
+  if (N < 2 || D_in < 1 || D_out < 1) return 0;
+  return probe_layout(N, D_in, D_out).total;
+}
+
+rmm_status rmm_variance_probe(const void* X, const void* dY, int64_t N, int64_t D_in, int64_t D_out, int64_t B_proj,
+                              rmm_dist dist, rmm_dtype dt, double* out, void* dW_exact, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+  if (N < 2) return RMM_ERR_INVALID_ARG;                       // Eq. 9 divides by N - 1
+  rmm_status st = check_common(N, D_in, D_out, B_proj, dist, dt);
+  if (st != RMM_OK) return st;
+  if (dt != RMM_DTYPE_BF16) return RMM_ERR_UNSUPPORTED;
+  if (!X || !dY || !out) return RMM_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(dY) || !aligned16(out) || !aligned16(dW_exact)) return RMM_ERR_INVALID_ARG;
+  const ProbeWorkspace w = probe_layout(N, D_in, D_out);
+  if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) != 0 || workspace_bytes < w.total)
+    return RMM_ERR_WORKSPACE;
+  if (!device_state().ok) return RMM_ERR_CUDA;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  int* status = reinterpret_cast<int*>(ws + w.status_off);
+  double* row_partial = reinterpret_cast<double*>(ws + w.row_off);
+  double* gemm_partial = reinterpret_cast<double*>(ws + w.gemm_off);
+  void* dw = dW_exact ? dW_exact : static_cast<void*>(ws + w.dw_off);
+  if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return RMM_ERR_CUDA;
+  row_norms_kernel<<<w.row_blocks, VAR_THREADS, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(X),
+                                                             reinterpret_cast<const __nv_bfloat16*>(dY), N, D_in, D_out,
+                                                             row_partial);
+  if (cudaGetLastError() != cudaSuccess) return RMM_ERR_CUDA;
+  // exact gradient dW* = dY^T X (Eq. 3) on the tensor cores; its epilogue leaves |dW*|_F^2 in gemm_partial
+  st = launch_tc<tc::A_MN, tc::B_MN>(dY, X, dw, nullptr, D_out, D_in, N, 1.0f, status, stream, gemm_partial);
+  if (st != RMM_OK) return st;
+  variance_finish_kernel<<<1, 32, 0, stream>>>(row_partial, w.row_blocks, gemm_partial, tc_grid_ctas(D_out, D_in) * tc::NEPI,
+                                              N, B_proj, (int)dist, out);
+  return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
 
 rmm_status rmm_bias_grad_static(const void* dY, int64_t N, int64_t D_out, rmm_dtype dt, void* db, void* cuda_stream) {

@@ -62,6 +62,8 @@ struct GemmParams {
   const void* bias;   // bf16 [N] or nullptr
   float alpha;
   int* status;        // workspace status word
+  double* sumsq;      // nullptr, or [gridDim.x][NEPI]: every epilogue warp adds up the squares of the (scaled,
+                      // biased, unrounded) results it converts, for |C|_F^2 (variance diagnostics)
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -229,6 +231,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (lane == 0) tma_prefetch_desc(&tmC);
     int it = 0;
     uint32_t nbox = 0;                            // boxes filled so far: box nbox & 1 is next
+    double sq = 0.0;                              // this lane's share of |C|_F^2 (only with p.sumsq)
     for (int tile = pair; tile < num_tiles; tile += num_pairs, ++it) {
       const int buf = it & 1;
       const bool acc_ready =
@@ -263,6 +266,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
               }
             }
+            if (p.sumsq) {                        // rows and columns out of range hold exact zeros (zero-filled operands)
+#pragma unroll
+              for (int i = 0; i < 8; ++i) sq += (double)f[i] * (double)f[i];
+            }
             // row `lane` of the box, 16-byte chunk 4h + g, at its swizzled position
             const uint32_t dst = box + row_off + ((((uint32_t)(4 * h + g)) ^ sw) << 4);
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(pack_bf16x2(f[0], f[1])),
@@ -282,6 +289,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(accempty_leader0 + 8u * buf);
+    }
+    if (p.sumsq) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      if (lane == 0) p.sumsq[(size_t)blockIdx.x * NEPI + (warp - 2)] = sq;
     }
     if (lane == 0) bulk_wait_group_all();         // the boxes must outlive their stores
     __syncwarp();

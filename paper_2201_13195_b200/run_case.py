@@ -22,6 +22,7 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--forward-only", action="store_true")
+    ap.add_argument("--variance-probe", action="store_true", help="run rmm_variance_probe instead of the layer")
     a = ap.parse_args()
     td = torch.bfloat16 if a.dtype == "bf16" else torch.float32
     dist = P.RMM_DIST_GAUSSIAN if a.dist == "gaussian" else P.RMM_DIST_RADEMACHER
@@ -36,6 +37,18 @@ def main():
     dW = torch.empty(a.d_out, a.d_in, device="cuda", dtype=td)
     db = torch.empty(a.d_out, device="cuda", dtype=td)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if a.variance_probe:
+        pws = torch.empty(P.rmm_variance_probe_workspace_bytes(a.n, a.d_in, a.d_out), dtype=torch.uint8, device="cuda")
+        out = torch.empty(8, dtype=torch.float64, device="cuda")
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(a.reps):
+            P.rmm_variance_probe(X, dY, a.k, dist, out=out, workspace=pws)
+        e1.record()
+        torch.cuda.synchronize()
+        assert P.rmm_last_device_status(pws) == P.RMM_OK
+        print(f"{e0.elapsed_time(e1) / a.reps:.4f} ms per probe;", dict(zip(P.VARIANCE_FIELDS, out.cpu().tolist())))
+        return
     torch.cuda.synchronize()
     e0.record()
     for i in range(a.reps):

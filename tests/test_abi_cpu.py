@@ -150,3 +150,28 @@ def test_rmm_linear_bproj_rule_matches_harness_rule():
     from paper_2201_13195_b200.rmm_linear import bproj_from_rho
     for n, rho in ((4096, 0.1), (4096, 0.2), (4096, 0.5), (4096, 0.9), (16384, 0.1), (512, 0.5), (7, 0.01), (3, 1.0)):
         assert bproj_from_rho(n, rho) == R.bproj_from_rho(n, rho) >= 1
+
+
+def test_variance_probe_argument_errors(lib):
+    i64, vp = C.c_int64, C.c_void_p
+    probe = lib.rmm_variance_probe
+    probe.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, C.c_int, vp, vp, vp, C.c_size_t, vp]
+    size = lib.rmm_variance_probe_workspace_bytes
+    size.argtypes = [i64, i64, i64]
+    size.restype = C.c_size_t
+    assert size(1, 8, 8) == 0 and size(16, 0, 8) == 0
+    need = size(4096, 768, 3072)
+    assert need >= 3072 * 768 * 2          # room for the exact gradient when the caller does not want it
+    p = 4096
+    INVALID, UNSUPPORTED, WORKSPACE, CUDA = 1, 2, 3, 4
+    assert probe(p, p, 1, 8, 8, 1, 0, 0, p, None, p, 1 << 30, None) == INVALID         # N < 2: Eq. 9 divides by N - 1
+    assert probe(None, p, 16, 8, 8, 4, 0, 0, p, None, p, 1 << 30, None) == INVALID     # null X
+    assert probe(p, p, 16, 8, 8, 4, 0, 0, None, None, p, 1 << 30, None) == INVALID     # null out
+    assert probe(p, p, 16, 8, 8, 17, 0, 0, p, None, p, 1 << 30, None) == INVALID       # B_proj > N
+    assert probe(p, p, 16, 8, 8, 4, 0, 1, p, None, p, 1 << 30, None) == UNSUPPORTED    # fp32 tensors
+    assert probe(p, p, 16, 12, 8, 4, 0, 0, p, None, p, 1 << 30, None) == UNSUPPORTED   # D_in % 8
+    assert probe(p, p, 16, 8, 8, 4, 0, 0, p, None, p, 64, None) == WORKSPACE           # too small
+    assert probe(p, p, 16, 8, 8, 4, 0, 0, p, None, None, 0, None) == WORKSPACE
+    import torch
+    if not torch.cuda.is_available():
+        assert probe(p, p, 16, 8, 8, 4, 0, 0, p, None, p, 1 << 30, None) == CUDA        # no device: an error, no fallback
