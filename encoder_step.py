@@ -18,10 +18,13 @@ import torch.nn.functional as F
 
 class Config:
     def __init__(self, hidden=768, heads=12, ffn=3072, layers=12, vocab=50265, max_pos=514, classes=2, dropout=0.1,
-                 rho=0.2, dist="gaussian"):
+                 rho=0.2, dist="gaussian", fused_qkv=False):
         self.hidden, self.heads, self.ffn, self.layers = hidden, heads, ffn, layers
         self.vocab, self.max_pos, self.classes, self.dropout = vocab, max_pos, classes, dropout
         self.rho, self.dist = rho, dist
+        # fused_qkv: one hidden -> 3 hidden layer for Q, K and V.  As an RMM layer it draws one S and
+        # keeps one X_proj for the three projections, which all read the same input.
+        self.fused_qkv = fused_qkv
 
 
 ROBERTA_BASE = dict(hidden=768, heads=12, ffn=3072, layers=12)
@@ -41,12 +44,14 @@ class Block(torch.nn.Module):
     """Post-LayerNorm Transformer block: self-attention (q, k, v, o) and feed-forward (up, down)."""
 
     NAMES = ("q", "k", "v", "o", "up", "down")
+    NAMES_FUSED = ("qkv", "o", "up", "down")
 
     def __init__(self, cfg, kind, index, workspace):
         super().__init__()
         h, f = cfg.hidden, cfg.ffn
-        shapes = {"q": (h, h), "k": (h, h), "v": (h, h), "o": (h, h), "up": (h, f), "down": (f, h)}
-        for i, name in enumerate(self.NAMES):
+        shapes = {"q": (h, h), "k": (h, h), "v": (h, h), "qkv": (h, 3 * h), "o": (h, h), "up": (h, f), "down": (f, h)}
+        self.names = self.NAMES_FUSED if cfg.fused_qkv else self.NAMES
+        for i, name in enumerate(self.names):
             setattr(self, name, _make_linear(kind, *shapes[name], cfg, 6 * index + i + 1, workspace))
         self.ln1 = torch.nn.LayerNorm(h, device="cuda", dtype=torch.bfloat16)
         self.ln2 = torch.nn.LayerNorm(h, device="cuda", dtype=torch.bfloat16)
@@ -55,8 +60,11 @@ class Block(torch.nn.Module):
     def forward(self, x):
         b, s, h = x.shape
         split = lambda t: t.view(b, s, self.heads, h // self.heads).transpose(1, 2)
-        a = F.scaled_dot_product_attention(split(self.q(x)), split(self.k(x)), split(self.v(x)),
-                                           dropout_p=self.p if self.training else 0.0)
+        if len(self.names) == 4:
+            q, k, v = self.qkv(x).split(h, dim=-1)
+        else:
+            q, k, v = self.q(x), self.k(x), self.v(x)
+        a = F.scaled_dot_product_attention(split(q), split(k), split(v), dropout_p=self.p if self.training else 0.0)
         a = self.o(a.transpose(1, 2).reshape(b, s, h))
         x = self.ln1(x + F.dropout(a, self.p, self.training))
         y = self.down(F.gelu(self.up(x)))
@@ -90,8 +98,8 @@ class Encoder(torch.nn.Module):
         return self.head_out(torch.tanh(self.head_dense(x[:, 0]))).float()
 
     def block_linears(self):
-        """[(name, module)] of the 6 * layers linear layers inside the blocks, in forward order."""
-        return [(f"block{i}.{n}", getattr(b, n)) for i, b in enumerate(self.blocks) for n in Block.NAMES]
+        """[(name, module)] of the linear layers inside the blocks (6 per block, 4 with fused QKV), in forward order."""
+        return [(f"block{i}.{n}", getattr(b, n)) for i, b in enumerate(self.blocks) for n in b.names]
 
 
 def copy_weights(dst: Encoder, src: Encoder):
@@ -191,8 +199,9 @@ def main():
     ap.add_argument("--dist", default="gaussian", choices=["gaussian", "rademacher"])
     ap.add_argument("--batch", type=int, default=32)
     ap.add_argument("--seq", type=int, default=128)
+    ap.add_argument("--fused-qkv", action="store_true", help="one 768 -> 2304 layer (one S, one X_proj) for Q, K, V")
     a = ap.parse_args()
-    cfg = Config(**ROBERTA_BASE, rho=a.rho, dist=a.dist)
+    cfg = Config(**ROBERTA_BASE, rho=a.rho, dist=a.dist, fused_qkv=a.fused_qkv)
     res = {}
     for kind in ("rmm", "exact"):
         res[kind] = measure(kind, cfg, a.batch, a.seq, a.steps, max(a.warmup, 3))
@@ -203,7 +212,8 @@ def main():
             "value": res["rmm"]["ms_per_step"], "higher_is_better": False, "n_gpus": 1, "steps": a.steps,
             "warmup": max(a.warmup, 3), "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "roberta_base_encoder", "layers": cfg.layers, "hidden": cfg.hidden, "ffn": cfg.ffn,
-                       "batch": a.batch, "seq": a.seq, "rho": a.rho, "sketch": a.dist, "optimizer": "AdamW (fused)"},
+                       "batch": a.batch, "seq": a.seq, "rho": a.rho, "sketch": a.dist, "optimizer": "AdamW (fused)",
+                       "fused_qkv": a.fused_qkv},
             "exact_linear_ms": res["exact"]["ms_per_step"],
             "saved_activation_bytes": {
                 "block_linear_inputs_rmm": res["rmm"]["saved_bytes_block_linear_inputs"],

@@ -49,6 +49,25 @@ def test_small_encoder_every_layer_matches_oracle():
         assert torch.equal(m.bias.grad, m.trace[0]["db"])
 
 
+def test_fused_qkv_layer_matches_oracle_and_saves_one_sketch():
+    """Q, K and V as one 3x-wide RMM layer: one S and one X_proj for the three projections."""
+    import encoder_step as E
+    cfg = E.Config(hidden=64, heads=2, ffn=128, layers=1, vocab=300, dropout=0.0, rho=0.25, fused_qkv=True)
+    torch.manual_seed(4)
+    model = E.Encoder(cfg, "rmm").train()
+    names = [n for n, _ in model.block_linears()]
+    assert names == ["block0.qkv", "block0.o", "block0.up", "block0.down"]
+    for _, m in model.block_linears():
+        m.trace = []
+    ids, labels = E.make_batch(7, batch=3, seq=40, vocab=cfg.vocab)
+    E.train_step(model, None, ids, labels)
+    torch.cuda.synchronize()
+    qkv = dict(model.block_linears())["block0.qkv"]
+    assert qkv.trace[0]["X_proj"].shape == (30, 64) and qkv.trace[0]["Y"].shape == (120, 192)
+    for name, m in model.block_linears():
+        _check_trace_against_oracle(m.trace[0], name)
+
+
 def test_identity_sketch_reproduces_exact_linear_gradients():
     """With S = I (B_proj = N) the layer is the plain linear layer: every parameter gradient of the
     step must equal the one of the same model built from torch.nn.Linear."""
