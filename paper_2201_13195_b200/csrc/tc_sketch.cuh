@@ -612,10 +612,14 @@ __host__ __device__ inline long long sketch_partial_index(int r, int col) {
 }
 
 // Adds the partial tiles of each output tile in schedule order, scales, rounds to bf16.
-// grid = (tile groups * C, 16 column chunks), block = 128 threads: thread t owns row t of the
-// tile and the 32 columns of the chunk; blockIdx.x = C * tile group + rank of the CTA that
-// produced the 512-column block.  The loads of a thread are independent of each other.
-constexpr int SKR_CHUNK = 32;        // columns per block of the reduce kernel
+// grid = (tile groups * C, 32 column chunks), block = 128 threads: thread t owns row t of the
+// tile and the 16 columns of the chunk; blockIdx.x = C * tile group + rank of the CTA that
+// produced the 512-column block.  The kernel is bound by the latency of its loads (a few tens of
+// MB, mostly out of L2), so a thread fetches its 16 columns of four partial tiles at a time (16
+// independent 16-byte loads in flight) and then adds them in schedule order: the sum is the same
+// fixed sequence of fp32 additions whatever the batching.
+constexpr int SKR_CHUNK = 16;        // columns per block of the reduce kernel
+constexpr int SKR_BATCH = 4;         // partial tiles fetched together
 __global__ void __launch_bounds__(SK_BM)
 sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ ones_out) {
   const SketchSchedule& sc = p.sched;
@@ -627,18 +631,40 @@ sketch_reduce_kernel(SketchParams p, float scale, __nv_bfloat16* __restrict__ ou
   const long long j = m0 + r;
   const int col0 = blockIdx.y * SKR_CHUNK;
   if (j >= p.rows || n0 + col0 >= p.cols) return;
-  float4 acc[SKR_CHUNK / 4];
+  constexpr int Q = SKR_CHUNK / 4;      // float4 per thread and partial tile
+  float4 acc[Q];
 #pragma unroll
-  for (int g = 0; g < SKR_CHUNK / 4; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int g = 0; g < Q; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
   const long long off = sketch_partial_index(r, col0);
+  const float* pending[SKR_BATCH];
+  int npending = 0;
+  auto flush = [&]() {
+    float4 v[SKR_BATCH][Q];
+#pragma unroll
+    for (int b = 0; b < SKR_BATCH; ++b) {
+      if (b < npending) {
+#pragma unroll
+        for (int g = 0; g < Q; ++g) v[b][g] = __ldcs(reinterpret_cast<const float4*>(pending[b] + (long long)g * SK_BM * 4));
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < SKR_BATCH; ++b) {
+      if (b < npending) {
+#pragma unroll
+        for (int g = 0; g < Q; ++g) { acc[g].x += v[b][g].x; acc[g].y += v[b][g].y; acc[g].z += v[b][g].z; acc[g].w += v[b][g].w; }
+      }
+    }
+    npending = 0;
+  };
   sketch_for_each_slot_of_tile(sc, tile, [&](long long slot_index) {
     const float* src = p.partial + (slot_index * per_tile + rank) * (long long)SK_TILE_ELEMS + off;
-    float4 v[SKR_CHUNK / 4];
+    // constant indices only, so that the array stays in registers
 #pragma unroll
-    for (int g = 0; g < SKR_CHUNK / 4; ++g) v[g] = __ldcs(reinterpret_cast<const float4*>(src + (long long)g * SK_BM * 4));
-#pragma unroll
-    for (int g = 0; g < SKR_CHUNK / 4; ++g) { acc[g].x += v[g].x; acc[g].y += v[g].y; acc[g].z += v[g].z; acc[g].w += v[g].w; }
+    for (int b = 0; b < SKR_BATCH; ++b)
+      if (b == npending) pending[b] = src;
+    if (++npending == SKR_BATCH) flush();
   });
+  flush();
   const bool is_ones = p.ones_row && j == p.b_proj;
   const float s = is_ones ? 1.0f : scale;
   __nv_bfloat16* dst = is_ones ? ones_out : out + j * p.cols;
