@@ -189,7 +189,7 @@ int tc_grid_ctas(int64_t M, int64_t N) {
 
 template <int AMODE, int BMODE>
 rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, int64_t M, int64_t N, int64_t K,
-                     float alpha, int* status, cudaStream_t stream, double* sumsq = nullptr) {
+                     float alpha, int* status, cudaStream_t stream, double* sumsq = nullptr, bool clear_status = false) {
   CUtensorMap tmA, tmB, tmC;
   bool ok = make_tmap(&tmC, c, M, N, 32);        // store boxes of the epilogue: [32 rows][64 columns]
   if (AMODE == tc::A_K) ok &= make_tmap(&tmA, a, M, K, tc::BM);
@@ -199,7 +199,7 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   if (!ok) return RMM_ERR_CUDA;
   tc::GemmParams p;
   p.M = M; p.N = N; p.K = K;
-  p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.status = status; p.sumsq = sumsq;
+  p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.status = status; p.sumsq = sumsq; p.clear_status = clear_status ? 1 : 0;
   const int64_t tiles = ((N + tc::BN - 1) / tc::BN) * ((M + tc::PAIR_M - 1) / tc::PAIR_M);
   const int max_pairs = device_state().gemm_pairs;
   cudaLaunchConfig_t cfg = {};
@@ -219,7 +219,8 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
 // Sketch contraction out[j][d] = c * sum_n P[n][j] * b[n][d] for j < k (b is [tokens][cols] bf16),
 // and, when ones_out is given, ones_out[d] = sum_n b[n][d] from the extra row of ones.
 rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, int64_t cols, int64_t tokens, float c,
-                         int dist, const PhiloxKey& pk, float* partial, int* status, cudaStream_t stream) {
+                         int dist, const PhiloxKey& pk, float* partial, int* status, cudaStream_t stream,
+                         bool clear_status = false) {
   CUtensorMap tmB;
   const bool slab_map = cols % 64 == 0;
   if (!(slab_map ? make_tmap_slabs(&tmB, b, tokens, cols, tc::SK_BK, tc::SK_BN / 64)
@@ -235,6 +236,7 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   p.dist = dist;
   p.ones_row = ones_out ? 1 : 0;
   p.status = status;
+  p.clear_status = clear_status ? 1 : 0;
   const int C = tc::sketch_cluster_size(cols);
   p.sched = tc::make_sketch_schedule(p.rows, cols, tokens, C, device_state().sketch_clusters[C]);
   const int per_tile = C;
@@ -353,20 +355,21 @@ rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, i
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   char* ws = reinterpret_cast<char*>(workspace);
   int* status = reinterpret_cast<int*>(ws + w.status_off);
-  if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return RMM_ERR_CUDA;
   const PhiloxKey pk = make_philox_key(seed);
   const float c = sketch_scale(B_proj, dist);
 
   if (dt == RMM_DTYPE_BF16) {
+    // the first kernel of the call resets the status word (no separate memset on the stream)
     if (Y) {
       ScopedTiming t(RMM_STEP_Y, stream);
-      st = launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, status, stream);
+      st = launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, status, stream, nullptr, true);
       if (st != RMM_OK) return st;
     }
     ScopedTiming t(RMM_STEP_SKETCH, stream);
     return launch_sketch(X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, reinterpret_cast<float*>(ws + w.scratch_off),
-                         status, stream);
+                         status, stream, Y == nullptr);
   }
+  if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return RMM_ERR_CUDA;
   if (Y) {
     ScopedTiming t(RMM_STEP_Y, stream);
     st = simt_gemm_f32(false, X, D_in, 1, W, D_in, 1, Y, b, N, D_out, D_in, 1.0f, 0, pk, stream);
@@ -391,26 +394,27 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
   char* ws = reinterpret_cast<char*>(workspace);
   int* status = reinterpret_cast<int*>(ws + w.status_off);
   void* G = ws + w.g_off;
-  if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return RMM_ERR_CUDA;
   const PhiloxKey pk = make_philox_key(seed);
   const float c = sketch_scale(B_proj, dist);
 
   if (dt == RMM_DTYPE_BF16) {
+    // the first kernel of the call resets the status word (no separate memset on the stream)
     if (dX) {
       ScopedTiming t(RMM_STEP_DX, stream);
-      st = launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, status, stream);
+      st = launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, status, stream, nullptr, true);
       if (st != RMM_OK) return st;
     }
     {
       // db = dY^T 1 comes out of the same contraction as the extra row of ones of S^T
       ScopedTiming t(RMM_STEP_SDY, stream);
       st = launch_sketch(dY, G, db, B_proj, D_out, N, c, dist, pk, reinterpret_cast<float*>(ws + w.scratch_off), status,
-                         stream);
+                         stream, dX == nullptr);
       if (st != RMM_OK) return st;
     }
     ScopedTiming t(RMM_STEP_DW, stream);
     return launch_tc<tc::A_MN, tc::B_MN>(G, X_proj, dW, nullptr, D_out, D_in, B_proj, 1.0f, status, stream);
   }
+  if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return RMM_ERR_CUDA;
   if (dX) {
     ScopedTiming t(RMM_STEP_DX, stream);
     st = simt_gemm_f32(false, dY, D_out, 1, W, 1, D_in, dX, nullptr, N, D_in, D_out, 1.0f, 0, pk, stream);

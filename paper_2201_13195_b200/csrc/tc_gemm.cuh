@@ -62,6 +62,7 @@ struct GemmParams {
   const void* bias;   // bf16 [N] or nullptr
   float alpha;
   int* status;        // workspace status word
+  int clear_status;   // first kernel of a call: reset the status word (a timeout can only be recorded seconds later)
   double* sumsq;      // nullptr, or [gridDim.x][NEPI]: every epilogue warp adds up the squares of the (scaled,
                       // biased, unrounded) results it converts, for |C|_F^2 (variance diagnostics)
 };
@@ -90,6 +91,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   MBAR_PEEK_DECLARE();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();       // 0 = leader of the pair
+  if (p.clear_status && blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0;
   const bool leader = rank == 0;
   // Persistent: this pair takes pair tiles pair, pair + num_pairs, ...  Tile t is
   // (m = t / tiles_n, n = t % tiles_n): the pairs of one wave share a few A row blocks (the large,

@@ -270,6 +270,7 @@ struct SketchParams {
   int ones_row;
   int slab_map;        // tmB is the 3-D (column in slab, token, slab) view: needs cols % 64 == 0
   int* status;
+  int clear_status;    // first kernel of a call: reset the status word
   SketchSchedule sched;
 };
 
@@ -341,6 +342,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
   const uint32_t rank = (C == 1) ? 0u : cluster_ctarank();
   const SketchSchedule& sc = p.sched;
   const int cl = (int)(blockIdx.x / C);          // cluster index = worker index of the schedule
+  if (p.clear_status && blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < SK_A_STAGES; ++s) {
