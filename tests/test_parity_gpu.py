@@ -70,6 +70,9 @@ CASES = [
     ("multi_tile_ragged_f32", R.DTYPE_F32, 150, 70, 130, 66, R.DIST_RADEMACHER),
     ("rho_one_gauss", R.DTYPE_BF16, 200, 72, 136, 200, R.DIST_GAUSSIAN),
     ("k_multiple_of_tile", R.DTYPE_BF16, 512, 128, 256, 256, R.DIST_GAUSSIAN),
+    # dX has 38 x 2 = 76 tiles of 256 x 256: more than the 74 CTA pairs, so two pairs take a second tile
+    # (both accumulator buffers in use), with ragged last rows: 9700 = 37 * 256 + 228
+    ("dx_second_wave", R.DTYPE_BF16, 9700, 512, 64, 16, R.DIST_RADEMACHER),
 ]
 
 
