@@ -199,7 +199,7 @@ def _sampled_full_size(name, n_samples=48):
 
 
 @pytest.mark.parametrize("name", ["base_ffn_up_rho0.2", "base_ffn_down_rad_rho0.2", "base_qkv_rad_rho0.2",
-                                  "large_ffn_up_rho0.1", "large_ffn_down_rho0.1"])
+                                  "large_ffn_up_rho0.1", "large_ffn_down_rho0.1", "large_ffn_up_k1663_aligned"])
 def test_full_size_sampled(name):
     assert _sampled_full_size(name)
 
