@@ -199,7 +199,7 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   if (!ok) return RMM_ERR_CUDA;
   tc::GemmParams p;
   p.M = M; p.N = N; p.K = K;
-  p.C = c; p.ldc = N; p.bias = bias; p.alpha = alpha; p.status = status; p.sumsq = sumsq; p.clear_status = clear_status ? 1 : 0;
+  p.bias = bias; p.alpha = alpha; p.status = status; p.sumsq = sumsq; p.clear_status = clear_status ? 1 : 0;
   const int64_t tiles = ((N + tc::BN - 1) / tc::BN) * ((M + tc::PAIR_M - 1) / tc::PAIR_M);
   const int max_pairs = device_state().gemm_pairs;
   cudaLaunchConfig_t cfg = {};

@@ -57,8 +57,6 @@ enum : int { B_K = 0, B_MN = 1 };
 
 struct GemmParams {
   int64_t M, N, K;
-  void* C;            // bf16 [M][ldc]
-  int64_t ldc;
   const void* bias;   // bf16 [N] or nullptr
   float alpha;
   int* status;        // workspace status word
