@@ -35,6 +35,7 @@ DEFAULT_WORKLOAD = "large_ffn_up_rho0.1"
 NCU_DRAM_BYTES = {("large_ffn_up_rho0.1", "sdy"): (34.200832e6 / 4096, 14.971136e6)}
 
 STEP_ORDER = ("y", "sketch", "dx", "sdy", "dw", "db")
+E2E_LANES = 3    # streams (each with its own staging buffers and thread) that take the end-to-end steps in turn
 
 
 def load_peaks():
@@ -204,7 +205,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(R.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--e2e-steps", type=int, default=30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--reference-budget-s", type=float, default=90.0,
                     help="wall-clock budget of the whole --impl reference run (sizes its token sample)")
@@ -309,27 +310,56 @@ def main():
     # ---- end to end through the host-buffer entry points (pinned host memory)
     e2e = None
     if rank == 0 or world > 1:
+        # E2E_LANES lanes (stream, device staging, workspace, host result buffers) take the steps in turn, so that
+        # the host->device copies of one step overlap the device->host copies of the step before it (the two
+        # copy directions are separate engines); every step still copies all its inputs in and all its results out.
         hX, hW, hdY = [torch.from_numpy(a).to(td).pin_memory() for a in (X, W, dY)]
-        hY, hXp = torch.empty_like(Y, device="cpu").pin_memory(), torch.empty_like(Xp, device="cpu").pin_memory()
-        hdX, hdW, hdb = [torch.empty_like(a, device="cpu").pin_memory() for a in (dX, dW, db)]
         nb = max(P.rmm_host_staging_bytes(N, w.d_in, w.d_out, k, w.dtype, bw, o) for bw in (0, 1) for o in (0, 1))
-        dev_in = torch.empty(nb, dtype=torch.uint8, device="cuda")
-        dev_out = torch.empty(nb, dtype=torch.uint8, device="cuda")
+        lanes = []
+        for li in range(E2E_LANES):
+            ln = {"stream": stream if li == 0 else torch.cuda.Stream(),
+                  "hY": torch.empty_like(Y, device="cpu").pin_memory(), "hXp": torch.empty_like(Xp, device="cpu").pin_memory(),
+                  "hd": [torch.empty_like(a, device="cpu").pin_memory() for a in (dX, dW, db)],
+                  "dev_in": torch.empty(nb, dtype=torch.uint8, device="cuda"),
+                  "dev_out": torch.empty(nb, dtype=torch.uint8, device="cuda"),
+                  "ws": ws if li == 0 else P.alloc_workspace(N, w.d_in, w.d_out, k, w.dtype)}
+            lanes.append(ln)
 
         def e2e_step(i):
+            ln = lanes[i % E2E_LANES]
             seed = w.seed + 100000 + i
-            P.rmm_forward_host(hX, hW, None, seed, k, w.dist, hY, hXp, dev_in, dev_out, ws, stream=stream)
-            P.rmm_backward_host(hdY, hW, hXp, seed, w.dist, hdX, hdW, hdb, dev_in, dev_out, ws, stream=stream)
+            P.rmm_forward_host(hX, hW, None, seed, k, w.dist, ln["hY"], ln["hXp"], ln["dev_in"], ln["dev_out"], ln["ws"],
+                               stream=ln["stream"])
+            P.rmm_backward_host(hdY, hW, ln["hXp"], seed, w.dist, *ln["hd"], ln["dev_in"], ln["dev_out"], ln["ws"],
+                                stream=ln["stream"])
 
-        for i in range(2):
+        for i in range(2 * E2E_LANES):
             e2e_step(i)
+        torch.cuda.synchronize()
         barrier()
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        g0.record(stream)
-        for i in range(args.e2e_steps):
-            e2e_step(2 + i)
-        g1.record(stream)
+        g0.record(lanes[0]["stream"])
+        for ln in lanes[1:]:
+            ln["stream"].wait_event(g0)               # no lane starts before the start mark
+        # The host entry points return when their results are in host memory, so each lane runs in its own
+        # thread (ctypes releases the interpreter lock during the call).
+        def lane_worker(li):
+            for i in range(li, args.e2e_steps, E2E_LANES):
+                e2e_step(2 * E2E_LANES + i)
+
+        workers = [threading.Thread(target=lane_worker, args=(li,)) for li in range(E2E_LANES)]
+        for t in workers:
+            t.start()
+        for t in workers:
+            t.join()
+        for ln in lanes[1:]:                          # the end mark follows the last step of every lane
+            done = torch.cuda.Event()
+            done.record(ln["stream"])
+            lanes[0]["stream"].wait_event(done)
+        g1.record(lanes[0]["stream"])
         torch.cuda.synchronize()
+        for ln in lanes:
+            assert P.rmm_last_device_status(ln["ws"]) == P.RMM_OK
         dt = g0.elapsed_time(g1) * 1e-3
         tt = torch.tensor([dt], dtype=torch.float64, device="cuda")
         if world > 1:
@@ -339,7 +369,8 @@ def main():
         h2d = (N * w.d_in + w.d_out * w.d_in) * eb + (N * w.d_out + w.d_out * w.d_in + k * w.d_in) * eb
         d2h = (N * w.d_out + k * w.d_in) * eb + (N * w.d_in + w.d_out * w.d_in + w.d_out) * eb
         e2e = {"value": world * fl["total"] * args.e2e_steps / dt / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "ms_per_step": 1e3 * dt / args.e2e_steps}
+               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "ms_per_step": 1e3 * dt / args.e2e_steps,
+               "streams": E2E_LANES}
 
     if rank == 0:
         cpu = None if args.no_cpu_baseline or world > 1 else cpu_baseline(w)
