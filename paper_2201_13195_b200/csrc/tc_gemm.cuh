@@ -21,7 +21,7 @@
 // them out of tensor memory, applies alpha and the bias, rounds to bf16, writes a [32 rows][128 B]
 // box into shared memory (128-byte swizzle) and hands it to a TMA store; two boxes per warp, so
 // the conversion of one overlaps the store of the other.  The stores reach L2 as whole 128-byte
-// lines (per-lane 16-byte stores of row fragments cost the Y GEMM a quarter of its time), and
+// lines (per-lane 16-byte stores of row fragments cost the Y GEMM a sixth of its time), and
 // the tensor map clips rows and columns beyond the matrix.
 //
 // Warp roles per CTA: warp 0 = TMA producer (its halves), warp 1 = tensor-memory owner and, in

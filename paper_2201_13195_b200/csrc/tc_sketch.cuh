@@ -32,6 +32,11 @@
 // accumulator (warp 1 owns the tensor memory); warps 3..14 generate S tiles, in three groups of
 // four that each own one ring stage, and drain the accumulator.  A ring: 3 stages of 64 tokens;
 // B ring: 5 stages of 32 tokens (the B ring is the latency-critical one: it holds 2.5 K-steps).
+// What limits the kernel: a 64-token step moves 80 KB of operands through shared memory, so the
+// two rings hold about 2.6 steps, less than the round trip MMA completion -> commit -> producer
+// -> (TMA load | stores + bulk copy to the peer) -> MMA issue.  With all generator arithmetic
+// or all B loads removed (experiments) the kernel is less than 10 % faster: neither the ALUs nor
+// L2 nor the tensor pipe (about 70 % busy in steady state) is the bound, the ring depth is.
 // Barriers of a CTA: fullA[s] (the group's warps + the bytes copied in by the other CTAs: the
 // stage is complete in this CTA's ring), emptyA[s] (2 C commits: every MMA warp of every CTA of
 // the cluster has consumed the stage, so it may be overwritten everywhere), fullB / emptyB (TMA
