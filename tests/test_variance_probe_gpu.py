@@ -58,3 +58,41 @@ def test_variance_probe_identity_sketch_has_no_variance():
     dY = torch.randn(64, 48, device="cuda").to(torch.bfloat16)
     out = P.rmm_variance_probe(X, dY, 64, P.RMM_DIST_IDENTITY).cpu().numpy()
     assert out[5] == 0.0 and out[0] > 0 and out[4] > 0
+
+
+@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER])
+def test_gpu_estimator_is_unbiased_and_has_the_probed_variance(dist):
+    """The library's own dW over many seeds: its mean is the exact gradient dY^T X (Section 2.2,
+    unbiasedness) and its mean squared error is the D^2_RMM that rmm_variance_probe reports for the
+    same X and dY (Lemma 2 with the fourth moment kept)."""
+    import paper_2201_13195_b200 as P
+    n, d_in, d_out, k, T = 96, 16, 24, 12, 3000
+    g = np.random.default_rng(11)
+    u = g.standard_normal((n, 1))      # a shared token factor: |X^T dY|^2 comparable to |X|^2 |dY|^2 (alpha about 0.5)
+    X = R.round_to_bf16((u @ g.standard_normal((1, d_in)) + 0.3 * g.standard_normal((n, d_in))).astype(np.float32))
+    dY = R.round_to_bf16((u @ g.standard_normal((1, d_out)) + 0.3 * g.standard_normal((n, d_out))).astype(np.float32))
+    Xd = torch.from_numpy(X).cuda().to(torch.bfloat16).contiguous()
+    dYd = torch.from_numpy(dY).cuda().to(torch.bfloat16).contiguous()
+    W = torch.zeros(d_out, d_in, dtype=torch.bfloat16, device="cuda")
+    ws = P.alloc_workspace(n, d_in, d_out, k, P.RMM_DTYPE_BF16)
+    Xp = torch.empty(k, d_in, dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty(d_out, d_in, dtype=torch.bfloat16, device="cuda")
+    exact = dY.astype(np.float64).T @ X.astype(np.float64)
+    acc = torch.zeros(d_out, d_in, dtype=torch.float64, device="cuda")
+    acc2 = torch.zeros(d_out, d_in, dtype=torch.float64, device="cuda")
+    ex = torch.from_numpy(exact).cuda()
+    for seed in range(T):
+        P.rmm_forward(Xd, W, None, 1000 + seed, k, dist, X_proj=Xp, workspace=ws, want_y=False)
+        P.rmm_backward(dYd, W, Xp, 1000 + seed, dist, dW=dW, workspace=ws, want_dx=False, want_db=False)
+        e = dW.double() - ex
+        acc += e
+        acc2 += e * e
+    torch.cuda.synchronize()
+    mean_err, mse = (acc / T).cpu().numpy(), float(acc2.sum().item()) / T
+    probe = P.rmm_variance_probe(Xd, dYd, k, dist).cpu().numpy()
+    # per-entry standard error of the mean; bf16 storage of X_proj, G and dW adds a bias far below it
+    se = np.sqrt(np.maximum((acc2 / T).cpu().numpy() - mean_err ** 2, 1e-30) / T)
+    z = np.abs(mean_err) / se
+    assert (z > 4.5).mean() <= 0.01 and z.max() < 6.0, float(z.max())
+    assert abs(mse / probe[5] - 1.0) < 0.08, (mse, probe[5], probe[6])
+    assert probe[7] > 0.3 and mse > 1.5 * probe[6]       # Eq. 11 as printed (fourth moment dropped) is far below
