@@ -176,7 +176,7 @@ def run_reference(args, w):
 def workload_config(w):
     touched = (2 * w.n_tokens * (w.d_in + w.d_out) * 2 + 3 * w.d_in * w.d_out + 2 * w.b_proj * (w.d_in + w.d_out)) * w.elem_bytes
     return {"workload": w.name, "n_tokens": w.n_tokens, "d_in": w.d_in, "d_out": w.d_out, "rho": w.rho,
-            "b_proj": w.b_proj, "sketch": ("gaussian", "rademacher", "identity")[w.dist], "seed": w.seed,
+            "b_proj": w.b_proj, "sketch": ("gaussian", "rademacher", "identity", "sors_hadamard")[w.dist], "seed": w.seed,
             "l2": f"inputs larger than L2: about {touched / 1e6:.0f} MB of tensors touched per step, no flush"}
 
 

@@ -39,6 +39,15 @@
  *   RMM_DIST_RADEMACHER P = +-1 with probability 1/2 (Section 3.2): counter
  *                       (n >> 7, j, 0, 1) gives 128 bits, entry P[n][j] is -1 when
  *                       bit (n & 31) of word ((n & 127) >> 5) is set;
+ *   RMM_DIST_SORS_HADAMARD  subsampled orthonormal matrix with random signs (Section 2.2 names the
+ *                       family; the paper gives no construction, this one is this library's):
+ *                       P[n][j] = d_n * H[n][r_j] with H the Sylvester Hadamard matrix of the
+ *                       smallest power-of-two order >= N, H[n][r] = (-1)^popcount(n & r);
+ *                       d_n = -1 when bit (n & 31) of word ((n & 127) >> 5) of counter
+ *                       (n >> 7, 0, 0, 2) is set; r_j = first word of counter (j, 0, 0, 3)
+ *                       modulo the order (columns drawn with replacement, so E[S S^T] = I
+ *                       exactly).  The contraction is the same dense one as for the other
+ *                       distributions (no fast transform is applied);
  *   RMM_DIST_IDENTITY   S = I (needs B_proj == N; c = 1): the case in which the
  *                       layer reduces to the exact linear layer; meant for tests.
  * In bf16 mode P is rounded to bfloat16 (nearest even) before it is used.
@@ -62,7 +71,12 @@ typedef enum {
   RMM_ERR_TIMEOUT = 5      /* a device-side wait gave up; results of that call are invalid */
 } rmm_status;
 
-typedef enum { RMM_DIST_GAUSSIAN = 0, RMM_DIST_RADEMACHER = 1, RMM_DIST_IDENTITY = 2 } rmm_dist;
+typedef enum {
+  RMM_DIST_GAUSSIAN = 0,
+  RMM_DIST_RADEMACHER = 1,
+  RMM_DIST_IDENTITY = 2,
+  RMM_DIST_SORS_HADAMARD = 3
+} rmm_dist;
 typedef enum { RMM_DTYPE_BF16 = 0, RMM_DTYPE_F32 = 1 } rmm_dtype;
 
 /*
@@ -211,7 +225,8 @@ rmm_status rmm_bias_grad_static(const void* dY, int64_t N, int64_t D_out, rmm_dt
  * It needs X, so it is a debugging aid for a probed layer, not part of a training step that
  * wants the memory saving (the paper, too, probes single layers: Section 4.2).
  *   in : X, dY (device, bf16 only: RMM_ERR_UNSUPPORTED for RMM_DTYPE_F32), N >= 2,
- *        1 <= B_proj <= N, dist as in rmm_forward
+ *        1 <= B_proj <= N, dist as in rmm_forward except RMM_DIST_SORS_HADAMARD
+ *        (RMM_ERR_UNSUPPORTED: its variance has no closed form among the above)
  *   out: out = 8 doubles in DEVICE memory (16-byte aligned), written on the stream;
  *        dW_exact (nullable) = the exact gradient dY^T X [D_out, D_in] in bf16, which the
  *        probe computes on the way

@@ -13,7 +13,7 @@ import numpy as np
 
 from . import build as _build
 
-DIST_GAUSSIAN, DIST_RADEMACHER, DIST_IDENTITY = 0, 1, 2
+DIST_GAUSSIAN, DIST_RADEMACHER, DIST_IDENTITY, DIST_SORS = 0, 1, 2, 3
 STORE_BF16, STORE_F32 = 0, 1
 
 _lib = C.CDLL(_build.build())

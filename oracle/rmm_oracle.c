@@ -35,6 +35,7 @@
 #define ORACLE_DIST_GAUSSIAN 0
 #define ORACLE_DIST_RADEMACHER 1
 #define ORACLE_DIST_IDENTITY 2
+#define ORACLE_DIST_SORS 3
 #define ORACLE_STORE_BF16 0
 #define ORACLE_STORE_F32 1
 
@@ -150,7 +151,13 @@ float oracle_scale(int64_t k, int dist) {
  *   8*(n>>3) .. +7 of column j (word i gives tokens 2i and 2i+1).
  * Rademacher: counter (n>>7, j, 0, 1) -> 128 bits; token n takes bit (n&31) of
  *   word ((n&127)>>5); a set bit means -1.
- * Identity: P[n][j] = (n == j). */
+ * Identity: P[n][j] = (n == j).
+ * SORS (subsampled orthonormal with random signs; the paper names the family in
+ *   Section 2.2 and gives no construction, this one is the build's): with L the
+ *   smallest power of two >= N and H the Sylvester Hadamard matrix of order L,
+ *   H[n][r] = (-1)^popcount(n & r):  P[n][j] = d_n * H[n][r_j], where d_n = -1 when
+ *   bit (n&31) of word ((n&127)>>5) of counter (n>>7, 0, 0, 2) is set, and r_j is the
+ *   first word of counter (j, 0, 0, 3) modulo L. */
 void oracle_generate_p_cols(uint64_t seed, int64_t N, int64_t k, int64_t j0, int64_t j1,
                             int dist, int storage, float* out) {
   const int64_t w = j1 - j0;
@@ -176,6 +183,26 @@ void oracle_generate_p_cols(uint64_t seed, int64_t N, int64_t k, int64_t j0, int
           if (n < N) out[n * w + (j - j0)] = ze;
           if (n + 1 < N) out[(n + 1) * w + (j - j0)] = zo;
         }
+      }
+    }
+    return;
+  }
+  if (dist == ORACLE_DIST_SORS) {
+    uint64_t L = 1;
+    while (L < (uint64_t)N) L <<= 1;
+    for (int64_t j = j0; j < j1; ++j) {
+      uint32_t cj[4] = {(uint32_t)j, 0u, 0u, 3u}, rj[4];
+      oracle_philox4x32_10(cj, key, rj);
+      const uint64_t col = (uint64_t)rj[0] % L;
+      for (int64_t n = 0; n < N; ++n) {
+        uint32_t cn[4] = {(uint32_t)(n >> 7), 0u, 0u, 2u}, rn[4];
+        oracle_philox4x32_10(cn, key, rn);
+        const int t = (int)(n & 127);
+        const int d_neg = (int)((rn[t >> 5] >> (t & 31)) & 1u);
+        int ones = 0;                                   /* popcount(n & col), bit by bit */
+        for (uint64_t b = (uint64_t)n & col; b != 0; b >>= 1) ones += (int)(b & 1u);
+        const float h = (ones & 1) ? -1.0f : 1.0f;
+        out[n * w + (j - j0)] = d_neg ? -h : h;
       }
     }
     return;

@@ -234,6 +234,7 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   p.tokens = tokens;
   p.partial = partial;
   p.dist = dist;
+  p.sors_mask = sors_mask_for(tokens);
   p.ones_row = ones_out ? 1 : 0;
   p.status = status;
   p.clear_status = clear_status ? 1 : 0;
@@ -275,6 +276,7 @@ rmm_status simt_gemm_f32(bool gen_a, const void* A, int64_t a_sm, int64_t a_sk, 
   g.B = B; g.b_sn = b_sn; g.b_sk = b_sk;
   g.C = C; g.ldc = N; g.bias = bias;
   g.M = M; g.N = N; g.K = K; g.alpha = alpha; g.dist = dist;
+  g.sors_mask = sors_mask_for(K);      // generated A: K is the token count
   return gen_a ? launch_simt<float, true>(g, pk, stream) : launch_simt<float, false>(g, pk, stream);
 }
 
@@ -319,7 +321,9 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 rmm_status check_common(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rmm_dist dist, rmm_dtype dt) {
   if (N < 1 || D_in < 1 || D_out < 1 || k < 1 || k > N) return RMM_ERR_INVALID_ARG;
   if (N > (int64_t)1 << 31 || D_in > (int64_t)1 << 30 || D_out > (int64_t)1 << 30) return RMM_ERR_INVALID_ARG;
-  if (dist != RMM_DIST_GAUSSIAN && dist != RMM_DIST_RADEMACHER && dist != RMM_DIST_IDENTITY) return RMM_ERR_INVALID_ARG;
+  if (dist != RMM_DIST_GAUSSIAN && dist != RMM_DIST_RADEMACHER && dist != RMM_DIST_IDENTITY &&
+      dist != RMM_DIST_SORS_HADAMARD)
+    return RMM_ERR_INVALID_ARG;
   if (dt != RMM_DTYPE_BF16 && dt != RMM_DTYPE_F32) return RMM_ERR_INVALID_ARG;
   if (dist == RMM_DIST_IDENTITY && k != N) return RMM_ERR_INVALID_ARG;
   if (dt == RMM_DTYPE_BF16 && (D_in % 8 != 0 || D_out % 8 != 0)) return RMM_ERR_UNSUPPORTED;
@@ -440,7 +444,9 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
 rmm_status rmm_debug_generate_s(uint64_t seed, int64_t N, int64_t B_proj, rmm_dist dist, rmm_dtype dt, void* S_out,
                                 void* cuda_stream) {
   if (N < 1 || B_proj < 1 || B_proj > N || !S_out) return RMM_ERR_INVALID_ARG;
-  if (dist != RMM_DIST_GAUSSIAN && dist != RMM_DIST_RADEMACHER && dist != RMM_DIST_IDENTITY) return RMM_ERR_INVALID_ARG;
+  if (dist != RMM_DIST_GAUSSIAN && dist != RMM_DIST_RADEMACHER && dist != RMM_DIST_IDENTITY &&
+      dist != RMM_DIST_SORS_HADAMARD)
+    return RMM_ERR_INVALID_ARG;
   if (dt != RMM_DTYPE_BF16 && dt != RMM_DTYPE_F32) return RMM_ERR_INVALID_ARG;
   if (dist == RMM_DIST_IDENTITY && B_proj != N) return RMM_ERR_INVALID_ARG;
   if (!device_state().ok) return RMM_ERR_CUDA;
@@ -546,6 +552,7 @@ rmm_status rmm_variance_probe(const void* X, const void* dY, int64_t N, int64_t 
   rmm_status st = check_common(N, D_in, D_out, B_proj, dist, dt);
   if (st != RMM_OK) return st;
   if (dt != RMM_DTYPE_BF16) return RMM_ERR_UNSUPPORTED;
+  if (dist == RMM_DIST_SORS_HADAMARD) return RMM_ERR_UNSUPPORTED;   // no closed form for its variance here
   if (!X || !dY || !out) return RMM_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(dY) || !aligned16(out) || !aligned16(dW_exact)) return RMM_ERR_INVALID_ARG;
   const ProbeWorkspace w = probe_layout(N, D_in, D_out);

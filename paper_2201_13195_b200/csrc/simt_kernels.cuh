@@ -29,6 +29,7 @@ struct SimtGemmArgs {
   int64_t M, N, K;
   float alpha;
   int dist;                            // generated A only
+  uint32_t sors_mask;                  // dist 3: order of the Hadamard matrix - 1
 };
 
 constexpr int SIMT_BM = 64, SIMT_BN = 64, SIMT_BK = 16, SIMT_THREADS = 256;
@@ -62,6 +63,10 @@ simt_gemm_kernel(SimtGemmArgs g, PhiloxKey pk) {
           uint32_t w[4];
           rademacher_128(pk, (uint32_t)(n8 >> 7), (uint32_t)j, w);
           const uint32_t bits = w[(n8 & 127) >> 5] >> (n8 & 31);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) z[i] = ((bits >> i) & 1u) ? -1.0f : 1.0f;
+        } else if (g.dist == 3) {
+          const uint32_t bits = sors_sign_bits_8(pk, (uint32_t)n8, (uint32_t)j, g.sors_mask);
 #pragma unroll
           for (int i = 0; i < 8; ++i) z[i] = ((bits >> i) & 1u) ? -1.0f : 1.0f;
         } else {
@@ -155,7 +160,7 @@ __global__ void dump_sketch_kernel(PhiloxKey pk, int dist, int64_t N, int64_t k,
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= N * k) return;
   const int64_t n = idx / k, j = idx % k;
-  out[idx] = from_f32<T>(sketch_entry(pk, dist, n, j, sizeof(T) == 2));
+  out[idx] = from_f32<T>(sketch_entry(pk, dist, n, j, sizeof(T) == 2, sors_mask_for(N)));
 }
 
 // The normal transform applied to caller-given words (debug entry point).

@@ -276,6 +276,7 @@ struct SketchParams {
   int slab_map;        // tmB is the 3-D (column in slab, token, slab) view: needs cols % 64 == 0
   int* status;
   int clear_status;    // first kernel of a call: reset the status word
+  uint32_t sors_mask;  // dist 3: order of the Hadamard matrix - 1
   SketchSchedule sched;
 };
 
@@ -295,6 +296,8 @@ __device__ __forceinline__ uint4 sketch_chunk(const PhiloxKey& pk, const SketchP
     word = (t >> 5) == 2 ? w[2] : word;
     word = (t >> 5) == 3 ? w[3] : word;
     v = rademacher_8_bf16(word, (t & 31) >> 3);
+  } else if (p.dist == 3) {
+    v = rademacher_8_bf16(sors_sign_bits_8(pk, (uint32_t)tok8, (uint32_t)j, p.sors_mask), 0);
   } else {
     const long long d = j - tok8;
     uint32_t q0 = 0, q1 = 0, q2 = 0, q3 = 0;

@@ -18,14 +18,14 @@ def main():
     ap.add_argument("--d-in", type=int, default=1024)
     ap.add_argument("--d-out", type=int, default=4096)
     ap.add_argument("--k", type=int, default=410)
-    ap.add_argument("--dist", default="gaussian", choices=["gaussian", "rademacher"])
+    ap.add_argument("--dist", default="gaussian", choices=["gaussian", "rademacher", "sors"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--forward-only", action="store_true")
     ap.add_argument("--variance-probe", action="store_true", help="run rmm_variance_probe instead of the layer")
     a = ap.parse_args()
     td = torch.bfloat16 if a.dtype == "bf16" else torch.float32
-    dist = P.RMM_DIST_GAUSSIAN if a.dist == "gaussian" else P.RMM_DIST_RADEMACHER
+    dist = {"gaussian": P.RMM_DIST_GAUSSIAN, "rademacher": P.RMM_DIST_RADEMACHER, "sors": P.RMM_DIST_SORS_HADAMARD}[a.dist]
     g = torch.Generator(device="cuda").manual_seed(0)
     X = torch.randn(a.n, a.d_in, device="cuda", generator=g).to(td)
     W = (0.02 * torch.randn(a.d_out, a.d_in, device="cuda", generator=g)).to(td)

@@ -69,6 +69,7 @@ def test_argument_errors_are_reported_before_any_launch(lib):
     assert fwd(p, p, None, 8, 8, 8, 0, 9, 0, 0, p, p, p, 1 << 20, None) == INVALID          # B_proj > N
     assert fwd(p, p, None, 8, 8, 8, 0, 0, 0, 0, p, p, p, 1 << 20, None) == INVALID          # B_proj < 1
     assert fwd(p, p, None, 8, 8, 8, 0, 4, 5, 0, p, p, p, 1 << 20, None) == INVALID          # bad dist
+    assert fwd(p, p, None, 8, 8, 8, 0, 4, 3, 0, p, p, None, 0, None) == WORKSPACE           # dist 3 is valid: next check
     assert fwd(p, p, None, 8, 8, 8, 0, 4, 0, 3, p, p, p, 1 << 20, None) == INVALID          # bad dtype
     assert fwd(p, p, None, 8, 8, 8, 0, 4, 2, 0, p, p, p, 1 << 20, None) == INVALID          # identity needs k == N
     assert fwd(p + 4, p, None, 8, 8, 8, 0, 4, 0, 0, p, p, p, 1 << 20, None) == INVALID      # misaligned X
@@ -169,6 +170,7 @@ def test_variance_probe_argument_errors(lib):
     assert probe(p, p, 16, 8, 8, 4, 0, 0, None, None, p, 1 << 30, None) == INVALID     # null out
     assert probe(p, p, 16, 8, 8, 17, 0, 0, p, None, p, 1 << 30, None) == INVALID       # B_proj > N
     assert probe(p, p, 16, 8, 8, 4, 0, 1, p, None, p, 1 << 30, None) == UNSUPPORTED    # fp32 tensors
+    assert probe(p, p, 16, 8, 8, 4, 3, 0, p, None, p, 1 << 30, None) == UNSUPPORTED    # no closed form for the Hadamard sketch
     assert probe(p, p, 16, 12, 8, 4, 0, 0, p, None, p, 1 << 30, None) == UNSUPPORTED   # D_in % 8
     assert probe(p, p, 16, 8, 8, 4, 0, 0, p, None, p, 64, None) == WORKSPACE           # too small
     assert probe(p, p, 16, 8, 8, 4, 0, 0, p, None, None, 0, None) == WORKSPACE

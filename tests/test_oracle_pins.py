@@ -136,6 +136,30 @@ def test_rademacher_counter_mapping():
     assert np.array_equal(S, P.astype(np.float64) * float(np.float32(1) / np.sqrt(np.float32(k))))
 
 
+def test_sors_is_sign_flipped_hadamard_columns():
+    """P[n][j] = d_n * H[n][r_j]: H against scipy's Sylvester Hadamard matrix, d_n and r_j against the
+    independent Philox transcription; N not a power of two takes the first N rows of the next order."""
+    from scipy.linalg import hadamard
+    for seed, N, k in ((3, 64, 9), (0xABCDEF0123456789, 300, 5), (7, 1, 2), (11, 129, 4)):
+        L = 1
+        while L < N:
+            L *= 2
+        H = hadamard(L) if L > 1 else np.ones((1, 1))
+        key = [seed & M32, seed >> 32]
+        P = O.generate_p(seed, N, k, O.DIST_SORS, O.STORE_BF16)
+        assert set(np.unique(P)) <= {-1.0, 1.0}
+        d = np.array([-1.0 if (_philox_python([n >> 7, 0, 0, 2], key)[(n & 127) >> 5] >> (n & 31)) & 1 else 1.0
+                      for n in range(N)])
+        for j in range(k):
+            r = _philox_python([j, 0, 0, 3], key)[0] % L
+            assert np.array_equal(P[:, j], d * H[:N, r]), (seed, N, j)
+        S = O.generate_s(seed, N, k, O.DIST_SORS, O.STORE_F32)
+        assert np.array_equal(S, P.astype(np.float64) * float(np.float32(1) / np.sqrt(np.float32(k))))
+    # the full orthonormal matrix: all L columns of H, each once, give S S^T = I exactly (what subsampling draws from)
+    H = hadamard(32) / math.sqrt(32.0)
+    assert np.allclose(H @ H.T, np.eye(32), atol=1e-12)
+
+
 def test_identity_matrix():
     assert np.array_equal(O.generate_s(1, 6, 6, O.DIST_IDENTITY, O.STORE_BF16), np.eye(6))
 
@@ -208,7 +232,7 @@ def test_identity_sketch_reproduces_exact_gradient():
 
 
 # --------------------------------------------------------------- statistical properties
-@pytest.mark.parametrize("dist", [O.DIST_GAUSSIAN, O.DIST_RADEMACHER])
+@pytest.mark.parametrize("dist", [O.DIST_GAUSSIAN, O.DIST_RADEMACHER, O.DIST_SORS])
 def test_unbiasedness_of_s_st(dist):
     N, k, T = 16, 8, 4000
     acc = np.zeros((N, N))
@@ -220,6 +244,26 @@ def test_unbiasedness_of_s_st(dist):
     sd_diag = math.sqrt((2.0 if dist == O.DIST_GAUSSIAN else 0.0) / (k * T)) + 1e-6
     assert np.abs(np.diag(M) - 1.0).max() < 4.5 * sd_diag
     assert np.abs(off).max() < 4.5 * math.sqrt(1.0 / (k * T))
+
+
+def test_sors_gradient_is_unbiased():
+    """E_S[dW_rmm] = dW for the subsampled Hadamard sketch (token count not a power of two)."""
+    rng = np.random.default_rng(5)
+    N, Din, Dout, k, T = 6, 4, 3, 3, 20000
+    X = rng.standard_normal((N, Din))
+    dY = X[:, :Dout] * 0.8 + 0.4 * rng.standard_normal((N, Dout))
+    W = rng.standard_normal((Dout, Din))
+    dW_star = O.exact_dw(dY, X)
+    tot, sq = np.zeros_like(dW_star), np.zeros_like(dW_star)
+    for seed in range(T):
+        S = O.generate_s(500 + seed, N, k, O.DIST_SORS, O.STORE_F32)
+        _, Xp = O.forward(X, W, None, S, want_y=False)
+        _, dW, _, _ = O.backward(dY, W, Xp, S, want_dx=False, want_db=False)
+        tot += dW
+        sq += dW * dW
+    mean = tot / T
+    sd = np.sqrt(np.maximum(sq / T - mean**2, 0) / T)
+    assert (np.abs(mean - dW_star) / sd).max() < 4.5
 
 
 @pytest.mark.parametrize("dist", [O.DIST_GAUSSIAN, O.DIST_RADEMACHER])

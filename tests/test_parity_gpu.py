@@ -20,7 +20,7 @@ def _P():
 
 # ------------------------------------------------------------------ S bit-exact
 @pytest.mark.parametrize("dtype", [R.DTYPE_BF16, R.DTYPE_F32])
-@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER])
+@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS])
 @pytest.mark.parametrize("N,k,seed", [(37, 5, 0), (300, 130, 0xDEADBEEF12345678), (1024, 64, 3)])
 def test_sketch_dump_bit_exact(dtype, dist, N, k, seed):
     P = _P()
@@ -42,7 +42,7 @@ def test_gaussian_transform_bit_exact_on_all_radius_and_angle_inputs():
 
 
 @pytest.mark.parametrize("dtype", [R.DTYPE_BF16, R.DTYPE_F32])
-@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER])
+@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS])
 def test_production_kernel_sketch_bit_exact(dtype, dist):
     """X = I makes X_proj = c * P^T: the sketch kernel's own S, entry by entry."""
     P = _P()
@@ -70,6 +70,8 @@ CASES = [
     ("multi_tile_ragged_f32", R.DTYPE_F32, 150, 70, 130, 66, R.DIST_RADEMACHER),
     ("rho_one_gauss", R.DTYPE_BF16, 200, 72, 136, 200, R.DIST_GAUSSIAN),
     ("k_multiple_of_tile", R.DTYPE_BF16, 512, 128, 256, 256, R.DIST_GAUSSIAN),
+    ("sors_ragged_bf16", R.DTYPE_BF16, 389, 264, 520, 77, R.DIST_SORS),
+    ("sors_ragged_f32", R.DTYPE_F32, 150, 70, 130, 66, R.DIST_SORS),
     # dX has 38 x 2 = 76 tiles of 256 x 256: more than the 74 CTA pairs, so two pairs take a second tile
     # (both accumulator buffers in use), with ragged last rows: 9700 = 37 * 256 + 228
     ("dx_second_wave", R.DTYPE_BF16, 9700, 512, 64, 16, R.DIST_RADEMACHER),
@@ -199,7 +201,8 @@ def _sampled_full_size(name, n_samples=48):
 
 
 @pytest.mark.parametrize("name", ["base_ffn_up_rho0.2", "base_ffn_down_rad_rho0.2", "base_qkv_rad_rho0.2",
-                                  "large_ffn_up_rho0.1", "large_ffn_down_rho0.1", "large_ffn_up_k1663_aligned"])
+                                  "large_ffn_up_rho0.1", "large_ffn_down_rho0.1", "large_ffn_up_k1663_aligned",
+                                  "large_ffn_up_sors_rho0.1"])
 def test_full_size_sampled(name):
     assert _sampled_full_size(name)
 
