@@ -71,6 +71,15 @@ bool allow_big_smem(K kernel, int bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
+// The sketch kernel for a cluster size (1 or 2) and a distribution (rmm_dist value).
+typedef void (*SketchKernelFn)(const CUtensorMap, tc::SketchParams, PhiloxKey);
+SketchKernelFn sketch_kernel_fn(int c, int dist) {
+  static const SketchKernelFn table[2][4] = {
+      {tc::sketch_kernel<1, 0>, tc::sketch_kernel<1, 1>, tc::sketch_kernel<1, 2>, tc::sketch_kernel<1, 3>},
+      {tc::sketch_kernel<2, 0>, tc::sketch_kernel<2, 1>, tc::sketch_kernel<2, 2>, tc::sketch_kernel<2, 3>}};
+  return table[c == 2 ? 1 : 0][dist & 3];
+}
+
 // How many clusters of `c` CTAs of kernel `k` can be resident on the device at once.
 template <typename K>
 bool query_clusters(K k, int c, int* out, int threads = tc::SK_THREADS, int smem = tc::SK_SMEM_BYTES) {
@@ -109,14 +118,12 @@ DeviceState& device_state() {
     a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_K>, tc::GEMM_SMEM_BYTES);
     a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_MN>, tc::GEMM_SMEM_BYTES);
     a &= allow_big_smem(tc::gemm_kernel<tc::A_MN, tc::B_MN>, tc::GEMM_SMEM_BYTES);
-    a &= allow_big_smem(tc::sketch_kernel<1>, tc::SK_SMEM_BYTES);
-    a &= allow_big_smem(tc::sketch_kernel<2>, tc::SK_SMEM_BYTES);
-    a &= allow_big_smem(tc::sketch_kernel<4>, tc::SK_SMEM_BYTES);
+    for (int c = 1; c <= 2; ++c)
+      for (int d = 0; d < 4; ++d) a &= allow_big_smem(sketch_kernel_fn(c, d), tc::SK_SMEM_BYTES);
     if (a) {
       st.sketch_clusters[1] = st.num_sms < tc::SK_MAX_CTAS ? st.num_sms : tc::SK_MAX_CTAS;
-      a &= query_clusters(tc::sketch_kernel<2>, 2, &st.sketch_clusters[2]);
+      a &= query_clusters(tc::sketch_kernel<2, 0>, 2, &st.sketch_clusters[2]);   // the same for every distribution
       a &= query_clusters(tc::gemm_kernel<tc::A_K, tc::B_K>, 2, &st.gemm_pairs, 64 + 32 * tc::NEPI, tc::GEMM_SMEM_BYTES);
-      a &= query_clusters(tc::sketch_kernel<4>, 4, &st.sketch_clusters[4]);
     }
     st.ok = a;
   });
@@ -251,9 +258,7 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cudaError_t le = C == 4 ? cudaLaunchKernelEx(&cfg, tc::sketch_kernel<4>, tmB, p, pk)
-                 : C == 2 ? cudaLaunchKernelEx(&cfg, tc::sketch_kernel<2>, tmB, p, pk)
-                          : cudaLaunchKernelEx(&cfg, tc::sketch_kernel<1>, tmB, p, pk);
+  cudaError_t le = cudaLaunchKernelEx(&cfg, sketch_kernel_fn(C, dist), tmB, p, pk);
   if (le != cudaSuccess) return RMM_ERR_CUDA;
   dim3 rgrid((unsigned)(p.sched.tiles() * per_tile), tc::SK_BN / tc::SKR_CHUNK);
   tc::sketch_reduce_kernel<<<rgrid, tc::SK_BM, 0, stream>>>(p, c, reinterpret_cast<__nv_bfloat16*>(out),

@@ -12,7 +12,7 @@
 // Sharing S across a cluster.  Generating the normals is plain ALU work (about 24
 // instructions each) and takes about as many issue slots as the MMAs that consume them take
 // tensor cycles.  CTAs that compute the same sketch rows for neighbouring 512-column blocks
-// therefore form a thread-block cluster of C (1 or 2; 4 compiles but too few such clusters are
+// therefore form a thread-block cluster of C (1 or 2; with 4 too few such clusters are
 // co-resident): each CTA generates 128/C rows of every S^T stage into its own operand ring and
 // sends that block to the other CTAs with one bulk shared-to-shared copy each, counted on the
 // destination's full barrier, so each generated entry feeds C x 512 columns.  Every CTA runs
@@ -281,13 +281,15 @@ struct SketchParams {
 };
 
 // Eight consecutive tokens (tok8 a multiple of 8) of sketch row j as packed bf16: one 16-byte
-// chunk of the operand tile.
+// chunk of the operand tile.  The distribution is a compile-time parameter: a run-time dispatch in
+// this innermost routine costs the Gaussian path registers and about 2 % of the kernel's time.
+template <int DIST>
 __device__ __forceinline__ uint4 sketch_chunk(const PhiloxKey& pk, const SketchParams& p, long long j, long long tok8) {
   constexpr uint32_t kOnes = 0x3f803f80u;   // two bf16 1.0
   uint4 v;
-  if (p.dist == 0) {
+  if (DIST == 0) {
     v = gaussian_8_bf16(pk, (uint32_t)tok8, (uint32_t)j);
-  } else if (p.dist == 1) {
+  } else if (DIST == 1) {
     uint32_t w[4];
     rademacher_128(pk, (uint32_t)(tok8 >> 7), (uint32_t)j, w);
     const int t = (int)(tok8 & 127);
@@ -296,7 +298,7 @@ __device__ __forceinline__ uint4 sketch_chunk(const PhiloxKey& pk, const SketchP
     word = (t >> 5) == 2 ? w[2] : word;
     word = (t >> 5) == 3 ? w[3] : word;
     v = rademacher_8_bf16(word, (t & 31) >> 3);
-  } else if (p.dist == 3) {
+  } else if (DIST == 3) {
     v = rademacher_8_bf16(sors_sign_bits_8(pk, (uint32_t)tok8, (uint32_t)j, p.sors_mask), 0);
   } else {
     const long long d = j - tok8;
@@ -315,7 +317,7 @@ __device__ __forceinline__ uint4 sketch_chunk(const PhiloxKey& pk, const SketchP
 // Layout of an S^T stage (128 rows x 64 tokens): K-major with the 128-byte swizzle: row r at
 // byte 128 r, its 16-byte chunk c (tokens 8c .. 8c+7) stored at chunk position c ^ (r & 7).
 
-template <int C>
+template <int C, int DIST>
 __global__ void __launch_bounds__(SK_THREADS, 1)
 sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey pk) {
   extern __shared__ uint8_t smem_raw[];
@@ -543,7 +545,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
         for (int it = 0; it < TASKS_PER_THREAD; ++it) {
           const int t = it * GROUP_THREADS + gtid;
           const int r = (int)rank * (SK_BM / C) + (t >> 3), c = t & 7;
-          v[it] = sketch_chunk(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
+          v[it] = sketch_chunk<DIST>(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
           off[it] = (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
         }
         const bool freed = (C == 1) ? mbar_wait_warp(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)
