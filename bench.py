@@ -29,10 +29,10 @@ METRIC = "RMM linear fwd+bwd TFLOP/s (bf16)"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "large_ffn_up_rho0.1"
 # (workload, step) -> (dram__bytes_read.sum per token row of the kernel's input, dram__bytes_write.sum
-# per launch), from an ncu capture of sketch_kernel<2> at 4096 tokens: 34.20 MB read (the dY stream, in
-# proportion to the tokens), 14.97 MB written (fp32 partial tiles that leave L2; their number follows
+# per launch), from an ncu capture of sketch_kernel<2> at 4096 tokens: 33.70 MB read (the dY stream, in
+# proportion to the tokens), 14.68 MB written (fp32 partial tiles that leave L2; their number follows
 # the schedule, not the token count).
-NCU_DRAM_BYTES = {("large_ffn_up_rho0.1", "sdy"): (34.200832e6 / 4096, 14.971136e6)}
+NCU_DRAM_BYTES = {("large_ffn_up_rho0.1", "sdy"): (33.698304e6 / 4096, 14.677504e6)}
 
 STEP_ORDER = ("y", "sketch", "dx", "sdy", "dw", "db")
 E2E_LANES = 3    # streams (each with its own staging buffers and thread) that take the end-to-end steps in turn
@@ -304,7 +304,7 @@ def main():
     ncu_traffic = NCU_DRAM_BYTES.get((w.name, dom))
     if ncu_traffic is not None:
         roofline["traffic"] = ncu_traffic[0] * w.n_tokens + ncu_traffic[1]
-        roofline["traffic_note"] = ("dram read+write of sketch_kernel<2>: ncu at 4096 tokens, reads scaled by tokens, "
+        roofline["traffic_note"] = ("dram read+write of sketch_kernel<2,0>: ncu at 4096 tokens, reads scaled by tokens, "
                                     "writes (partial tiles) as captured")
 
     # ---- end to end through the host-buffer entry points (pinned host memory)
