@@ -1,5 +1,5 @@
 """One training step of a random-init RoBERTa-base-shaped encoder whose six linear layers per
-block are RMM layers (the paper's experimental model, Section 4: all linear layers of the
+block are RMM layers (the paper's experimental model, Section 3: all linear layers of the
 Transformer blocks are replaced).
 
 The harness around the layer is stock PyTorch (embeddings, scaled-dot-product attention,

@@ -36,10 +36,10 @@
  *                       Box-Muller transform on its two 16-bit halves evaluated with
  *                       a fixed sequence of correctly rounded fp32 operations, the
  *                       entries P[8*(n>>3) + 2i][j] and P[8*(n>>3) + 2i + 1][j];
- *   RMM_DIST_RADEMACHER P = +-1 with probability 1/2 (Section 3.2): counter
+ *   RMM_DIST_RADEMACHER P = +-1 with probability 1/2 (Section 3.5): counter
  *                       (n >> 7, j, 0, 1) gives 128 bits, entry P[n][j] is -1 when
  *                       bit (n & 31) of word ((n & 127) >> 5) is set;
- *   RMM_DIST_SORS_HADAMARD  subsampled orthonormal matrix with random signs (Section 2.2 names the
+ *   RMM_DIST_SORS_HADAMARD  subsampled orthonormal matrix with random signs (Section 2.1 names the
  *                       family; the paper gives no construction, this one is this library's):
  *                       P[n][j] = d_n * H[n][r_j] with H the Sylvester Hadamard matrix of the
  *                       smallest power-of-two order >= N, H[n][r] = (-1)^popcount(n & r);
@@ -223,7 +223,7 @@ rmm_status rmm_bias_grad_static(const void* dY, int64_t N, int64_t D_out, rmm_dt
  *            (it drops the fourth moment; it equals out[5] only when X^T dY = 0)
  *   out[7] = alpha = out[3] / (out[0] out[1])                               (Theorem 1, Eq. 13)
  * It needs X, so it is a debugging aid for a probed layer, not part of a training step that
- * wants the memory saving (the paper, too, probes single layers: Section 4.2).
+ * wants the memory saving (the paper, too, probes single layers: Section 3.3).
  *   in : X, dY (device, bf16 only: RMM_ERR_UNSUPPORTED for RMM_DTYPE_F32), N >= 2,
  *        1 <= B_proj <= N, dist as in rmm_forward except RMM_DIST_SORS_HADAMARD
  *        (RMM_ERR_UNSUPPORTED: its variance has no closed form among the above)

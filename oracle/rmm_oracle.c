@@ -153,7 +153,7 @@ float oracle_scale(int64_t k, int dist) {
  *   word ((n&127)>>5); a set bit means -1.
  * Identity: P[n][j] = (n == j).
  * SORS (subsampled orthonormal with random signs; the paper names the family in
- *   Section 2.2 and gives no construction, this one is the build's): with L the
+ *   Section 2.1 and gives no construction; this one is defined here): with L the
  *   smallest power of two >= N and H the Sylvester Hadamard matrix of order L,
  *   H[n][r] = (-1)^popcount(n & r):  P[n][j] = d_n * H[n][r_j], where d_n = -1 when
  *   bit (n&31) of word ((n&127)>>5) of counter (n>>7, 0, 0, 2) is set, and r_j is the

@@ -1,5 +1,5 @@
 """One training step of an encoder built from RMM linear layers (the paper's experimental model,
-Section 4): every block linear, with the activations and gradients the step actually produces,
+Section 3): every block linear, with the activations and gradients the step actually produces,
 is checked against the CPU oracle; the autograd wiring is checked against stock linears."""
 import numpy as np
 import pytest

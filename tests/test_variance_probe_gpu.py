@@ -62,7 +62,7 @@ def test_variance_probe_identity_sketch_has_no_variance():
 
 @pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER])
 def test_gpu_estimator_is_unbiased_and_has_the_probed_variance(dist):
-    """The library's own dW over many seeds: its mean is the exact gradient dY^T X (Section 2.2,
+    """The library's own dW over many seeds: its mean is the exact gradient dY^T X (Section 2.1,
     unbiasedness) and its mean squared error is the D^2_RMM that rmm_variance_probe reports for the
     same X and dY (Lemma 2 with the fourth moment kept)."""
     import paper_2201_13195_b200 as P
