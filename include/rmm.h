@@ -46,8 +46,10 @@
  *                       d_n = -1 when bit (n & 31) of word ((n & 127) >> 5) of counter
  *                       (n >> 7, 0, 0, 2) is set; r_j = first word of counter (j, 0, 0, 3)
  *                       modulo the order (columns drawn with replacement, so E[S S^T] = I
- *                       exactly).  The contraction is the same dense one as for the other
- *                       distributions (no fast transform is applied);
+ *                       exactly).  In bf16 mode, for 128 <= order <= 16384, the sketches are
+ *                       applied by a two-level Walsh-Hadamard transform over the token index
+ *                       (O(N D log N)); otherwise by the same dense contraction as the other
+ *                       distributions.  S is the same matrix either way;
  *   RMM_DIST_IDENTITY   S = I (needs B_proj == N; c = 1): the case in which the
  *                       layer reduces to the exact linear layer; meant for tests.
  * In bf16 mode P is rounded to bfloat16 (nearest even) before it is used.

@@ -12,6 +12,7 @@
 #include "simt_kernels.cuh"
 #include "sketch_rng.cuh"
 #include "tc_gemm.cuh"
+#include "fwht_kernels.cuh"
 #include "tc_sketch.cuh"
 #include "variance_kernels.cuh"
 
@@ -225,9 +226,59 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
 
 // Sketch contraction out[j][d] = c * sum_n P[n][j] * b[n][d] for j < k (b is [tokens][cols] bf16),
 // and, when ones_out is given, ones_out[d] = sum_n b[n][d] from the extra row of ones.
+// The subsampled-Hadamard sketch by a two-level Walsh-Hadamard transform (fwht_kernels.cuh).  Returns
+// RMM_ERR_UNSUPPORTED when the shape is outside the fast path (the caller then takes the dense kernel).
+// scratch holds, in this order: the grouped column list, the per-block column sums, the stage-1 result
+// T for as many columns per round as fit.
+rmm_status launch_sors_fast(const void* b, void* out, void* ones_out, int64_t k, int64_t cols, int64_t tokens, float c,
+                            const PhiloxKey& pk, void* scratch, size_t scratch_bytes, int* status, cudaStream_t stream,
+                            bool clear_status) {
+  const uint32_t mask = sors_mask_for(tokens);
+  const int64_t L = (int64_t)mask + 1;
+  if (L < FW_ROWS || L > (int64_t)FW_ROWS * FW_ROWS) return RMM_ERR_UNSUPPORTED;
+  const int A = (int)(L / FW_ROWS);
+  uint8_t* base = reinterpret_cast<uint8_t*>(scratch);
+  size_t off = 0;
+  SorsGroups g;
+  g.offsets = reinterpret_cast<int*>(base + off);
+  off += align_up(129 * sizeof(int));
+  g.entries = reinterpret_cast<int2*>(base + off);
+  off += align_up((size_t)k * sizeof(int2));
+  if (off + 2 * kAlign >= scratch_bytes) return RMM_ERR_UNSUPPORTED;
+  const size_t per_col = (size_t)A * sizeof(float) + (size_t)L * 2;       // column sums + T, per column of a round
+  const int64_t cols64 = (cols + FW_COLS - 1) / FW_COLS * FW_COLS;
+  int64_t wslab = (int64_t)((scratch_bytes - off - 2 * kAlign) / per_col) / FW_COLS * FW_COLS;
+  if (wslab > cols64) wslab = cols64;
+  if (wslab < FW_COLS) return RMM_ERR_UNSUPPORTED;
+  float* colsum = reinterpret_cast<float*>(base + off);
+  off += align_up((size_t)A * (size_t)wslab * sizeof(float));
+  __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(base + off);
+  sors_group_kernel<<<1, 1024, 0, stream>>>(pk, k, mask, g, status, clear_status ? 1 : 0);
+  if (cudaGetLastError() != cudaSuccess) return RMM_ERR_CUDA;
+  const __nv_bfloat16* B = reinterpret_cast<const __nv_bfloat16*>(b);
+  __nv_bfloat16* O = reinterpret_cast<__nv_bfloat16*>(out);
+  __nv_bfloat16* ones = reinterpret_cast<__nv_bfloat16*>(ones_out);
+  for (int64_t c0 = 0; c0 < cols; c0 += wslab) {
+    const int width = (int)(cols - c0 < wslab ? cols - c0 : wslab);
+    const unsigned slabs = (unsigned)((width + FW_COLS - 1) / FW_COLS);
+    fwht_stage1_kernel<<<dim3(slabs, (unsigned)A), FW_THREADS, 0, stream>>>(B + c0, cols, tokens, width, pk, T, wslab,
+                                                                           ones ? colsum : nullptr);
+    if (cudaGetLastError() != cudaSuccess) return RMM_ERR_CUDA;
+    fwht_stage2_kernel<<<dim3(slabs, FW_ROWS), FW_THREADS, 0, stream>>>(T, wslab, A, width, g, c, O + c0, cols,
+                                                                       ones ? colsum : nullptr, ones ? ones + c0 : nullptr);
+    if (cudaGetLastError() != cudaSuccess) return RMM_ERR_CUDA;
+  }
+  return RMM_OK;
+}
+
 rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, int64_t cols, int64_t tokens, float c,
                          int dist, const PhiloxKey& pk, float* partial, int* status, cudaStream_t stream,
-                         bool clear_status = false) {
+                         bool clear_status = false, size_t scratch_bytes = 0) {
+  if (dist == RMM_DIST_SORS_HADAMARD && scratch_bytes > 0) {
+    const rmm_status fs = launch_sors_fast(b, out, ones_out, k, cols, tokens, c, pk, partial, scratch_bytes, status, stream,
+                                           clear_status);
+    if (fs != RMM_ERR_UNSUPPORTED) return fs;
+  }
   CUtensorMap tmB;
   const bool slab_map = cols % 64 == 0;
   if (!(slab_map ? make_tmap_slabs(&tmB, b, tokens, cols, tc::SK_BK, tc::SK_BN / 64)
@@ -376,7 +427,7 @@ rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, i
     }
     ScopedTiming t(RMM_STEP_SKETCH, stream);
     return launch_sketch(X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, reinterpret_cast<float*>(ws + w.scratch_off),
-                         status, stream, Y == nullptr);
+                         status, stream, Y == nullptr, w.total - w.scratch_off);
   }
   if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return RMM_ERR_CUDA;
   if (Y) {
@@ -417,7 +468,7 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
       // db = dY^T 1 comes out of the same contraction as the extra row of ones of S^T
       ScopedTiming t(RMM_STEP_SDY, stream);
       st = launch_sketch(dY, G, db, B_proj, D_out, N, c, dist, pk, reinterpret_cast<float*>(ws + w.scratch_off), status,
-                         stream, dX == nullptr);
+                         stream, dX == nullptr, w.total - w.scratch_off);
       if (st != RMM_OK) return st;
     }
     ScopedTiming t(RMM_STEP_DW, stream);

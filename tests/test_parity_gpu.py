@@ -72,6 +72,9 @@ CASES = [
     ("k_multiple_of_tile", R.DTYPE_BF16, 512, 128, 256, 256, R.DIST_GAUSSIAN),
     ("sors_ragged_bf16", R.DTYPE_BF16, 389, 264, 520, 77, R.DIST_SORS),
     ("sors_ragged_f32", R.DTYPE_F32, 150, 70, 130, 66, R.DIST_SORS),
+    ("sors_below_fast_path", R.DTYPE_BF16, 37, 24, 40, 5, R.DIST_SORS),          # Hadamard order 64: dense kernel
+    ("sors_one_block", R.DTYPE_BF16, 128, 64, 72, 128, R.DIST_SORS),             # order 128: one block, no second level
+    ("sors_many_blocks", R.DTYPE_BF16, 2100, 136, 200, 300, R.DIST_SORS),        # order 4096: 32 blocks, last ones empty
     # dX has 38 x 2 = 76 tiles of 256 x 256: more than the 74 CTA pairs, so two pairs take a second tile
     # (both accumulator buffers in use), with ragged last rows: 9700 = 37 * 256 + 228
     ("dx_second_wave", R.DTYPE_BF16, 9700, 512, 64, 16, R.DIST_RADEMACHER),
