@@ -250,6 +250,10 @@ rmm_status launch_sors_fast(const void* b, void* out, void* ones_out, int64_t k,
   int64_t wslab = (int64_t)((scratch_bytes - off - 2 * kAlign) / per_col) / FW_COLS * FW_COLS;
   if (wslab > cols64) wslab = cols64;
   if (wslab < FW_COLS) return RMM_ERR_UNSUPPORTED;
+  {   // rounds of equal width rather than full ones and a narrow last one
+    const int64_t rounds = (cols64 + wslab - 1) / wslab;
+    wslab = ((cols64 + rounds - 1) / rounds + FW_COLS - 1) / FW_COLS * FW_COLS;
+  }
   float* colsum = reinterpret_cast<float*>(base + off);
   off += align_up((size_t)A * (size_t)wslab * sizeof(float));
   __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(base + off);
