@@ -6,8 +6,8 @@
 //     T[a][rb][:]  = sum_b H128[b][rb] * d_n * B[128 a + b][:]          (stage 1, inside 128-token blocks)
 //     out[j][:]    = c * sum_a H_A[a][ra_j] * T[a][rb_j][:]             (stage 2, across the A = L/128 blocks)
 // where L is the order of the Hadamard matrix (128 <= L <= 16384 here; other sizes take the dense
-// kernel).  Both stages are the same shared-memory butterfly network on a [128 rows][64 columns]
-// tile; they are bound by HBM: stage 1 reads B and writes T (bf16), stage 2 reads T once and
+// kernel).  Both stages are the same butterfly network (registers, one pass through shared memory)
+// on a [128 rows][64 columns] tile; they are bound by HBM: stage 1 reads B and writes T (bf16), stage 2 reads T once and
 // writes only the B_proj rows that were drawn.  db (the column sums of B) is taken along in
 // stage 1 per block and added up over the blocks, in order, by the rb = 0 CTAs of stage 2.
 //
@@ -61,56 +61,32 @@ sors_group_kernel(PhiloxKey pk, int64_t k, uint32_t mask, SorsGroups g, int* sta
   }
 }
 
-// Walsh-Hadamard transform over the rows of a [128][65] fp32 tile, all 64 columns at once.  Thread
-// (rg, c) = (tid >> 6, tid & 63) takes the 32 rows 32 rg .. 32 rg + 31 of column c into registers
-// (optionally negating the rows whose bit is set in dbits, and returning their plain sum), does the
-// five stages over the low row bits there, writes them back, and after one barrier does the two
-// stages over the high row bits for eight of the low indices: 6 passes over the tile in shared
-// memory instead of 14.  `len` (a power of two <= 128) rows are transformed; rows >= len are not read.
-__device__ __forceinline__ float fwht_tile(float (*tile)[FW_COLS + 1], int len, int tid, const uint32_t* dbits) {
-  const int c = tid & 63, rg = tid >> 6;
-  float sum = 0.f;
-  const int low = len < 32 ? len : 32;           // rows per group that take part
-  if (rg * 32 < len) {
-    float x[32];
-    const uint32_t bits = dbits ? dbits[rg] : 0u;
+// The 128-point Walsh-Hadamard transform of a [128 rows][64 columns] tile, rows = 16 g + i.
+// A thread owns two adjacent columns (lane -> columns 2 lane, 2 lane + 1: a warp reads or writes
+// one 128-byte row segment per instruction) and, in phase 1, the 16 rows i = 0..15 of group g = its
+// warp: four butterfly stages in registers.  The tile then goes through shared memory once; in
+// phase 2 warp w takes the rows i = 2 w, 2 w + 1 of all eight groups: three stages over g.
+// Rows that do not exist are zeros: for the Sylvester matrix the first A outputs of the 128-point
+// transform of a zero-padded vector are its A-point transform, so one code path serves every A.
+__device__ __forceinline__ void wht16(float (&x)[16]) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      x[i] = i < low ? tile[rg * 32 + i][c] : 0.f;
-      sum += x[i];
-      if ((bits >> i) & 1u) x[i] = -x[i];
-    }
+  for (int h = 1; h < 16; h <<= 1) {
 #pragma unroll
-    for (int h = 1; h < 32; h <<= 1) {
-      if (h < low) {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          if ((i & h) == 0) { const float u = x[i], v = x[i + h]; x[i] = u + v; x[i + h] = u - v; }
-        }
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < 32; ++i)
-      if (i < low) tile[rg * 32 + i][c] = x[i];
+    for (int i = 0; i < 16; ++i)
+      if ((i & h) == 0) { const float u = x[i], v = x[i + h]; x[i] = u + v; x[i + h] = u - v; }
   }
-  __syncthreads();
-  if (len > 32) {
-    const int groups = len / 32;                  // 2 or 4
+}
+__device__ __forceinline__ void wht8(float (&y)[8]) {
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      const int i = rg * 8 + q;
-      float y0 = tile[i][c], y1 = tile[32 + i][c], y2 = groups == 4 ? tile[64 + i][c] : 0.f, y3 = groups == 4 ? tile[96 + i][c] : 0.f;
-      const float s0 = y0 + y1, d0 = y0 - y1;
-      if (groups == 4) {
-        const float s1 = y2 + y3, d1 = y2 - y3;
-        tile[i][c] = s0 + s1; tile[32 + i][c] = d0 + d1; tile[64 + i][c] = s0 - s1; tile[96 + i][c] = d0 - d1;
-      } else {
-        tile[i][c] = s0; tile[32 + i][c] = d0;
-      }
-    }
-    __syncthreads();
+  for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+    for (int g = 0; g < 8; ++g)
+      if ((g & h) == 0) { const float u = y[g], v = y[g + h]; y[g] = u + v; y[g + h] = u - v; }
   }
-  return sum;
+}
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
 }
 
 // Stage 1.  grid = (column slabs of 64, A blocks of 128 tokens).  B is [N][ldb] bf16 (this launch
@@ -118,48 +94,56 @@ __device__ __forceinline__ float fwht_tile(float (*tile)[FW_COLS + 1], int len, 
 __global__ void __launch_bounds__(FW_THREADS)
 fwht_stage1_kernel(const __nv_bfloat16* __restrict__ B, int64_t ldb, int64_t N, int width, PhiloxKey pk,
                    __nv_bfloat16* __restrict__ T, int64_t ldt, float* __restrict__ colsum) {
-  __shared__ float tile[FW_ROWS][FW_COLS + 1];
-  __shared__ uint32_t dbits[4];
-  const int tid = threadIdx.x;
+  __shared__ float2 tile[FW_ROWS][FW_COLS / 2];
+  __shared__ float2 part[FW_THREADS / 32][FW_COLS / 2];
+  const int tid = threadIdx.x, w = tid >> 5, lane = tid & 31;
   const int c0 = blockIdx.x * FW_COLS, a = blockIdx.y;
-  if (tid == 0) {
-    uint32_t w[4];
-    philox4x32_10(pk, (uint32_t)a, 0u, 0u, 2u, w);      // the 128 sign bits of this block: tokens 128 a .. 128 a + 127
-    dbits[0] = w[0]; dbits[1] = w[1]; dbits[2] = w[2]; dbits[3] = w[3];
-  }
-  __syncthreads();
-  // 128 rows x 8 chunks of 8 columns; four chunks per thread
-  for (int t = tid; t < FW_ROWS * 8; t += FW_THREADS) {
-    const int b = t >> 3, ch = t & 7;
-    const int64_t n = (int64_t)a * FW_ROWS + b;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (n < N && c0 + 8 * ch < width) v = __ldg(reinterpret_cast<const uint4*>(B + n * ldb + c0 + 8 * ch));
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  const int col = c0 + 2 * lane;
+  const bool in_cols = col < width;                       // width is a multiple of 8: a column pair is all in or all out
+  uint32_t dw[4];
+  philox4x32_10(pk, (uint32_t)a, 0u, 0u, 2u, dw);         // the 128 sign bits of tokens 128 a .. 128 a + 127
+  const uint32_t bits = (dw[w >> 1] >> ((w & 1) * 16)) & 0xffffu;   // those of rows 16 w .. 16 w + 15
+  float x0[16], x1[16];
+  uint32_t raw[16];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      tile[b][8 * ch + 2 * i] = __uint_as_float(w[i] << 16);
-      tile[b][8 * ch + 2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
+  for (int i = 0; i < 16; ++i) {
+    const int64_t n = (int64_t)a * FW_ROWS + 16 * w + i;
+    raw[i] = (in_cols && n < N) ? __ldg(reinterpret_cast<const uint32_t*>(B + n * ldb + col)) : 0u;
   }
-  __syncthreads();
-  __shared__ float part[4][FW_COLS];
-  const float psum = fwht_tile(tile, FW_ROWS, tid, dbits);     // signs d_n applied on the way in; psum = plain sum of 32 rows
-  if (colsum != nullptr) {                                      // column sums of the block, the four row groups in order
-    part[tid >> 6][tid & 63] = psum;
-    __syncthreads();
-    if (tid < FW_COLS && c0 + tid < width)
-      colsum[(int64_t)a * ldt + c0 + tid] = (part[0][tid] + part[1][tid]) + (part[2][tid] + part[3][tid]);
-  }
-  for (int t = tid; t < FW_ROWS * 8; t += FW_THREADS) {
-    const int rb = t >> 3, ch = t & 7;
-    if (c0 + 8 * ch >= width) continue;
-    uint32_t o[4];
+  float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      __nv_bfloat162 h = __floats2bfloat162_rn(tile[rb][8 * ch + 2 * i], tile[rb][8 * ch + 2 * i + 1]);
-      o[i] = *reinterpret_cast<uint32_t*>(&h);
+  for (int i = 0; i < 16; ++i) {
+    x0[i] = __uint_as_float(raw[i] << 16);
+    x1[i] = __uint_as_float(raw[i] & 0xffff0000u);
+    s0 += x0[i];
+    s1 += x1[i];
+    if ((bits >> i) & 1u) { x0[i] = -x0[i]; x1[i] = -x1[i]; }
+  }
+  wht16(x0);
+  wht16(x1);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) tile[16 * w + i][lane] = make_float2(x0[i], x1[i]);
+  part[w][lane] = make_float2(s0, s1);
+  __syncthreads();
+  if (colsum != nullptr && w == 0 && in_cols) {            // column sums of the block: the eight row groups in order
+    float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+    for (int g = 0; g < FW_THREADS / 32; ++g) { t0 += part[g][lane].x; t1 += part[g][lane].y; }
+    *reinterpret_cast<float2*>(colsum + (int64_t)a * ldt + col) = make_float2(t0, t1);
+  }
+#pragma unroll
+  for (int ii = 0; ii < 2; ++ii) {
+    const int i = 2 * w + ii;
+    float y0[8], y1[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) { const float2 v = tile[16 * g + i][lane]; y0[g] = v.x; y1[g] = v.y; }
+    wht8(y0);
+    wht8(y1);
+    if (in_cols) {
+#pragma unroll
+      for (int g = 0; g < 8; ++g)
+        *reinterpret_cast<uint32_t*>(T + ((int64_t)a * FW_ROWS + 16 * g + i) * ldt + col) = pack2_bf16(y0[g], y1[g]);
     }
-    *reinterpret_cast<uint4*>(T + ((int64_t)a * FW_ROWS + rb) * ldt + c0 + 8 * ch) = make_uint4(o[0], o[1], o[2], o[3]);
   }
 }
 
@@ -170,38 +154,51 @@ __global__ void __launch_bounds__(FW_THREADS)
 fwht_stage2_kernel(const __nv_bfloat16* __restrict__ T, int64_t ldt, int A, int width, SorsGroups g, float scale,
                    __nv_bfloat16* __restrict__ out, int64_t ldo, const float* __restrict__ colsum,
                    __nv_bfloat16* __restrict__ ones_out) {
-  __shared__ float tile[FW_ROWS][FW_COLS + 1];
-  const int tid = threadIdx.x;
+  __shared__ float2 tile[FW_ROWS][FW_COLS / 2];
+  const int tid = threadIdx.x, w = tid >> 5, lane = tid & 31;
   const int c0 = blockIdx.x * FW_COLS, rb = blockIdx.y;
+  const int col = c0 + 2 * lane;
+  const bool in_cols = col < width;
   const int j0 = g.offsets[rb], j1 = g.offsets[rb + 1];
   const bool do_db = (rb == 0 && colsum != nullptr && ones_out != nullptr);
   if (j0 == j1 && !do_db) return;
   if (j0 < j1) {
-    for (int t = tid; t < A * 8; t += FW_THREADS) {
-      const int a = t >> 3, ch = t & 7;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (c0 + 8 * ch < width) v = *reinterpret_cast<const uint4*>(T + ((int64_t)a * FW_ROWS + rb) * ldt + c0 + 8 * ch);
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float x0[16], x1[16];
+    uint32_t raw[16];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        tile[a][8 * ch + 2 * i] = __uint_as_float(w[i] << 16);
-        tile[a][8 * ch + 2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-      }
+    for (int i = 0; i < 16; ++i) {
+      const int a = 16 * w + i;
+      raw[i] = (in_cols && a < A) ? *reinterpret_cast<const uint32_t*>(T + ((int64_t)a * FW_ROWS + rb) * ldt + col) : 0u;
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { x0[i] = __uint_as_float(raw[i] << 16); x1[i] = __uint_as_float(raw[i] & 0xffff0000u); }
+    wht16(x0);
+    wht16(x1);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) tile[16 * w + i][lane] = make_float2(x0[i], x1[i]);
+    __syncthreads();
+    float y0[2][8], y1[2][8];
+#pragma unroll
+    for (int ii = 0; ii < 2; ++ii) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { const float2 v = tile[16 * q + 2 * w + ii][lane]; y0[ii][q] = v.x; y1[ii][q] = v.y; }
+      wht8(y0[ii]);
+      wht8(y1[ii]);
+    }
+    __syncthreads();                                         // everyone has read its inputs: the tile takes the outputs
+#pragma unroll
+    for (int ii = 0; ii < 2; ++ii) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) tile[16 * q + 2 * w + ii][lane] = make_float2(y0[ii][q], y1[ii][q]);
     }
     __syncthreads();
-    fwht_tile(tile, A, tid, nullptr);
-    // 8 threads per output row (8 columns each), 32 rows per pass
-    for (int e = j0 + (tid >> 3); e < j1; e += FW_THREADS / 8) {
+    // the drawn rows of this rb: one warp per entry and pass, a 4-byte store per lane
+    for (int e = j0 + w; e < j1; e += FW_THREADS / 32) {
       const int2 jr = g.entries[e];
-      const int ch = tid & 7;
-      if (c0 + 8 * ch >= width) continue;
-      uint32_t o[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        __nv_bfloat162 h = __floats2bfloat162_rn(tile[jr.y][8 * ch + 2 * i] * scale, tile[jr.y][8 * ch + 2 * i + 1] * scale);
-        o[i] = *reinterpret_cast<uint32_t*>(&h);
+      if (in_cols) {
+        const float2 v = tile[jr.y][lane];
+        *reinterpret_cast<uint32_t*>(out + (int64_t)jr.x * ldo + col) = pack2_bf16(v.x * scale, v.y * scale);
       }
-      *reinterpret_cast<uint4*>(out + (int64_t)jr.x * ldo + c0 + 8 * ch) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
   if (do_db && tid < FW_COLS && c0 + tid < width) {
