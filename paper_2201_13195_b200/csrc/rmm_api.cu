@@ -99,36 +99,51 @@ bool query_clusters(K k, int c, int* out, int threads = tc::SK_THREADS, int smem
   return true;
 }
 
+// Per-device set-up, done at the first call made with that device current: the shared-memory opt-in
+// of the kernels (a per-device function attribute) and the residency counts that size the grids.
+constexpr int kMaxDevices = 64;
+
+void init_device_state(DeviceState& st, int dev) {
+  int major = 0, minor = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return;
+  if (cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess) return;
+  if (major != 10) return;  // the kernels are sm_100a only; there is no other path
+  if (cudaDeviceGetAttribute(&st.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr)
+    return;
+  st.encode = reinterpret_cast<EncodeTiledFn>(fn);
+  bool a = true;
+  a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_K>, tc::GEMM_SMEM_BYTES);
+  a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_MN>, tc::GEMM_SMEM_BYTES);
+  a &= allow_big_smem(tc::gemm_kernel<tc::A_MN, tc::B_MN>, tc::GEMM_SMEM_BYTES);
+  for (int c = 1; c <= 2; ++c)
+    for (int d = 0; d < 4; ++d) a &= allow_big_smem(sketch_kernel_fn(c, d), tc::SK_SMEM_BYTES);
+  if (a) {
+    st.sketch_clusters[1] = st.num_sms < tc::SK_MAX_CTAS ? st.num_sms : tc::SK_MAX_CTAS;
+    a &= query_clusters(tc::sketch_kernel<2, 0>, 2, &st.sketch_clusters[2]);   // the same for every distribution
+    a &= query_clusters(tc::gemm_kernel<tc::A_K, tc::B_K>, 2, &st.gemm_pairs, 64 + 32 * tc::NEPI, tc::GEMM_SMEM_BYTES);
+  }
+  st.ok = a;
+}
+
+// State of the device that is current on the calling thread.  A device that cannot run the kernels (or an
+// index beyond kMaxDevices) yields a state with ok == false, and the entry points return RMM_ERR_CUDA.
 DeviceState& device_state() {
-  static DeviceState st;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    int dev = 0, major = 0, minor = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return;
-    if (cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess) return;
-    if (major != 10) return;  // the kernels are sm_100a only; there is no other path
-    if (cudaDeviceGetAttribute(&st.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess || fn == nullptr)
-      return;
-    st.encode = reinterpret_cast<EncodeTiledFn>(fn);
-    bool a = true;
-    a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_K>, tc::GEMM_SMEM_BYTES);
-    a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_MN>, tc::GEMM_SMEM_BYTES);
-    a &= allow_big_smem(tc::gemm_kernel<tc::A_MN, tc::B_MN>, tc::GEMM_SMEM_BYTES);
-    for (int c = 1; c <= 2; ++c)
-      for (int d = 0; d < 4; ++d) a &= allow_big_smem(sketch_kernel_fn(c, d), tc::SK_SMEM_BYTES);
-    if (a) {
-      st.sketch_clusters[1] = st.num_sms < tc::SK_MAX_CTAS ? st.num_sms : tc::SK_MAX_CTAS;
-      a &= query_clusters(tc::sketch_kernel<2, 0>, 2, &st.sketch_clusters[2]);   // the same for every distribution
-      a &= query_clusters(tc::gemm_kernel<tc::A_K, tc::B_K>, 2, &st.gemm_pairs, 64 + 32 * tc::NEPI, tc::GEMM_SMEM_BYTES);
-    }
-    st.ok = a;
-  });
-  return st;
+  static DeviceState states[kMaxDevices];
+  static bool tried[kMaxDevices] = {};
+  static DeviceState none;
+  static std::mutex mu;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return none;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!tried[dev]) {
+    tried[dev] = true;
+    init_device_state(states[dev], dev);
+  }
+  return states[dev];
 }
 
 // Tensor map of a row-major bf16 matrix [rows][cols] (cols contiguous), box = [box_rows][64 cols],
@@ -356,7 +371,6 @@ rmm_status launch_db(const void* dY, int64_t N, int64_t D_out, const Workspace& 
 // is only a host-side handle; kernels get the device address from cudaGetSymbolAddress.
 static __device__ __align__(256) float g_bias_grad_scratch[RMM_BIAS_GRAD_STATIC_SLICES * RMM_BIAS_GRAD_STATIC_MAX_D_OUT];
 
-constexpr int kMaxDevices = 64;
 float* g_bias_grad_scratch_addr[kMaxDevices] = {};
 std::mutex g_bias_grad_mutex;
 

@@ -85,7 +85,8 @@ WORKLOADS = {w.name: w for w in [
     # sketch rows plus the row of ones that carries db) fills whole 128-row tiles: 13 * 128 - 1.  Same tile count
     # and cost as B_proj = 1638, 1.5 % more sketch rows (lower variance); reported in addition, never instead.
     _w("large_ffn_up_k1663_aligned", DTYPE_BF16, 16384, 1024, 4096, 1663 / 16384, DIST_GAUSSIAN, 10, k_fixed=1663),
-    # the RoBERTa-large shape with the subsampled-Hadamard sketch (dense contraction, no fast transform)
+    # the RoBERTa-large shape with the subsampled-Hadamard sketch (in bf16 mode applied by the two-level Walsh-Hadamard
+    # transform; the dense contraction with the same S only outside Hadamard orders 128 .. 16384)
     _w("large_ffn_up_sors_rho0.1", DTYPE_BF16, 16384, 1024, 4096, 0.1, DIST_SORS, 11),
     # diagnostic: the RoBERTa-large shape with the cheap sketch distribution (isolates the cost of the normals)
     _w("large_ffn_up_rad_rho0.1", DTYPE_BF16, 16384, 1024, 4096, 0.1, DIST_RADEMACHER, 9),

@@ -15,18 +15,26 @@ def _np(t):
 
 
 def _check_trace_against_oracle(rec, name):
+    """Frobenius gate per tensor and the element-wise gate of tests/gpu_util.py on every element."""
     from oracle import oracle as O
+    import rmm_inputs as R
+    from tests.gpu_util import contraction_lengths, dw_operand_term, elementwise_excess
     X, W, dY = _np(rec["X"]), _np(rec["W"]), _np(rec["dY"])
     b = None if rec["b"] is None else _np(rec["b"])
     S = O.generate_s(rec["seed"], X.shape[0], rec["b_proj"], rec["dist"], O.STORE_BF16)
     Y, Xp = O.forward(X, W, b, S)
     got_xp = _np(rec["X_proj"])
-    dX, dW, db, _ = O.backward(dY, W, got_xp, S)     # stage-wise: backward gets the saved X_proj, as the library does
-    errs = {"Y": O.rel_frobenius(_np(rec["Y"]), Y), "X_proj": O.rel_frobenius(got_xp, Xp),
-            "dX": O.rel_frobenius(_np(rec["dX"]), dX), "dW": O.rel_frobenius(_np(rec["dW"]), dW),
-            "db": O.rel_frobenius(_np(rec["db"]), db)}
+    dX, dW, db, G = O.backward(dY, W, got_xp, S)     # stage-wise: backward gets the saved X_proj, as the library does
+    got = {"Y": _np(rec["Y"]), "X_proj": got_xp, "dX": _np(rec["dX"]), "dW": _np(rec["dW"]), "db": _np(rec["db"])}
+    ref = {"Y": Y, "X_proj": Xp, "dX": dX, "dW": dW, "db": db}
+    errs = {k: O.rel_frobenius(got[k], ref[k]) for k in ref}
     bad = {k: v for k, v in errs.items() if not v <= TOL}
     assert not bad, f"{name}: {bad} (all {errs})"
+    K = contraction_lengths(X.shape[0], X.shape[1], W.shape[0], rec["b_proj"])
+    for k in ref:
+        term = dw_operand_term(G, got_xp, R.DTYPE_BF16) if k == "dW" else None
+        ex, where = elementwise_excess(got[k], ref[k], R.DTYPE_BF16, K[k], term)
+        assert ex <= 1.0, f"{name}: {k}{list(where)} is {ex:.2f} x its element-wise bound"
     return errs
 
 

@@ -10,7 +10,8 @@ from oracle import oracle as O
 
 pytestmark = pytest.mark.gpu
 
-from tests.gpu_util import (STORE, TOL, TORCH_DTYPE, assert_parity, oracle_layer, run_layer, to_dev, to_np)  # noqa: E402
+from tests.gpu_util import (STORE, TOL, TORCH_DTYPE, assert_parity, contraction_lengths, dw_operand_term,  # noqa: E402
+                            elementwise_excess, oracle_layer, run_layer, to_dev, to_np)
 
 
 def _P():
@@ -58,6 +59,50 @@ def test_production_kernel_sketch_bit_exact(dtype, dist):
     assert np.array_equal(Xp.to(torch.float32).cpu().numpy(), want)
 
 
+def _selector(N, tokens, dtype):
+    """X [N, len(tokens)] with X[tokens[i]][i] = 1 and zeros elsewhere: X_proj[j][i] = c * P[tokens[i]][j] exactly
+    (one non-zero product per sum), so the production sketch kernel's own S can be compared bit for bit at the
+    chosen tokens without an N x N identity."""
+    X = torch.zeros((N, len(tokens)), dtype=TORCH_DTYPE[dtype], device="cuda")
+    X[torch.as_tensor(tokens, device="cuda"), torch.arange(len(tokens), device="cuda")] = 1.0
+    return X
+
+
+WIDE_S_CASES = [
+    # name, N, number of selected tokens (= D_in), k, seed
+    ("two_blocks_identity", 1024, 1024, 141, 78),        # X = I with two 512-column blocks: S stages shared by a CTA pair
+    ("four_blocks_many_steps", 4096, 2048, 300, 79),     # several column groups, 64 token steps, three row tiles
+    ("odd_blocks", 2000, 1536, 260, 80),                 # three 512-column blocks, ragged last token step
+    ("above_hadamard_fast_path", 16500, 1024, 141, 81),  # Hadamard order 32768: the dense kernel also for SORS
+]
+
+
+@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS])
+@pytest.mark.parametrize("case", WIDE_S_CASES, ids=[c[0] for c in WIDE_S_CASES])
+def test_production_kernel_sketch_bit_exact_wide(case, dist):
+    """S entry by entry on the launch shapes of the RoBERTa layers: results wider than one 512-column block
+    (stages of S^T exchanged inside a CTA pair or cluster), many token steps per tile, several row tiles."""
+    P = _P()
+    _, N, D, k, seed = case
+    rng = np.random.default_rng(seed)
+    if D == N:
+        tokens = np.arange(N)
+    else:   # first and last tokens, the edges of the 64-token steps, and random ones
+        edges = np.concatenate([np.arange(0, N, 64), np.arange(63, N, 64), [N - 1]])
+        rest = np.setdiff1d(np.arange(N), edges)
+        tokens = np.sort(np.concatenate([edges[:D // 2], rng.choice(rest, size=D - len(edges[:D // 2]), replace=False)]))
+    X = _selector(N, tokens, R.DTYPE_BF16)
+    W = torch.zeros((8, D), dtype=torch.bfloat16, device="cuda")
+    _, Xp = P.rmm_forward(X, W, None, seed, k, dist, want_y=False)
+    torch.cuda.synchronize()
+    Pm = O.generate_p(seed, N, k, dist, O.STORE_BF16)[tokens]          # [D, k] fp32
+    want = R.round_to_bf16((Pm.T * np.float32(O.scale(k, dist))).astype(np.float32))
+    got = Xp.to(torch.float32).cpu().numpy()
+    assert got.shape == want.shape
+    bad = np.argwhere(got != want)
+    assert bad.size == 0, f"{len(bad)} entries differ, first at sketch row {bad[0][0]}, token {tokens[bad[0][1]]}"
+
+
 # ------------------------------------------------------------------ whole layer, small and ragged
 CASES = [
     # name, dtype, N, D_in, D_out, k, dist
@@ -86,11 +131,12 @@ def test_layer_parity_small(case):
     name, dtype, N, Di, Do, k, dist = case
     w = R.small_case(name, dtype, N, Di, Do, k, dist, seed=len(name) * 1000003)
     got = run_layer(w)
+    K = contraction_lengths(N, Di, Do, k)
     ref = oracle_layer(w, got["inputs"], gpu_xproj=got["X_proj"])
-    assert_parity(got, ref, dtype)
+    assert_parity(got, ref, dtype, K=K)
     # end to end (oracle's own fp64 X_proj in backward)
     ref2 = oracle_layer(w, got["inputs"])
-    assert_parity(got, ref2, dtype, names=("dW",))
+    assert_parity(got, ref2, dtype, names=("dW",), K=K, end_to_end=True)
 
 
 def test_identity_sketch_is_exact_layer():
@@ -106,7 +152,7 @@ def test_fp32_config_parity():
     w = R.WORKLOADS["fp32_768x768_rho0.5"]
     got = run_layer(w)
     ref = oracle_layer(w, got["inputs"], gpu_xproj=got["X_proj"])
-    errs = assert_parity(got, ref, w.dtype)
+    errs = assert_parity(got, ref, w.dtype, K=contraction_lengths(w.n_tokens, w.d_in, w.d_out, w.b_proj))
     print("fp32 config errors", errs)
 
 
@@ -156,11 +202,17 @@ def test_host_buffer_entry_points():
     got = {"Y": hY.float().numpy(), "X_proj": hXp.float().numpy(), "dX": hdX.float().numpy(),
            "dW": hdW.float().numpy(), "db": hdb.float().numpy()}
     ref = oracle_layer(w, (X, W, b, dY), gpu_xproj=got["X_proj"].astype(np.float64))
-    assert_parity(got, ref, w.dtype)
+    assert_parity(got, ref, w.dtype, K=contraction_lengths(N, w.d_in, w.d_out, k))
 
 
 # ------------------------------------------------------------------ full-size workloads, sampled outputs
-def _sampled_full_size(name, n_samples=48):
+def _sampled_full_size(name):
+    """The launch configuration the benchmark times, checked on outputs the oracle computes one by one: one row
+    of Y and of dX in every 128-row block (every row block of every output tile), one row of X_proj in every
+    128-row sketch tile plus the first and last, one row of dW in every 128-row block, all of db; all columns of
+    each sampled row, so every column block of every tile is covered.  Expected values come from oracle.forward /
+    oracle.backward on the row subsets; each sampled row passes the Frobenius gate and every sampled element the
+    element-wise one."""
     P = _P()
     w = R.WORKLOADS[name]
     X, W, b, dY = R.make_inputs(w)
@@ -173,33 +225,43 @@ def _sampled_full_size(name, n_samples=48):
     assert P.rmm_last_device_status(ws) == P.RMM_OK
     rng = np.random.default_rng(1)
     X64, W64, dY64 = X.astype(np.float64), W.astype(np.float64), dY.astype(np.float64)
-    c = float(np.float32(O.scale(k, w.dist)))
+    K = contraction_lengths(N, Di, Do, k)
     tol = TOL[w.dtype]
 
-    def close(got, want, what):
+    def close(got, want, what, Klen, term=None):
         got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
         err = np.linalg.norm(got - want) / np.linalg.norm(want)
         assert err <= tol, (what, err)
+        for r in range(got.shape[0]):                      # every sampled row on its own as well
+            e = np.linalg.norm(got[r] - want[r]) / np.linalg.norm(want[r])
+            assert e <= tol, (what, r, e)
+        ex, where = elementwise_excess(got, want, w.dtype, Klen, term)
+        assert ex <= 1.0, (what, where, ex)
 
-    # Y and dX: sampled rows (full rows, so the Frobenius measure is over thousands of entries)
-    rows = rng.choice(N, size=8, replace=False)
-    close(to_np(Y[rows]), X64[rows] @ W64.T, "Y")
-    close(to_np(dX[rows]), dY64[rows] @ W64, "dX")
+    def one_per_block(total, block):
+        starts = np.arange(0, total, block)
+        return np.minimum(starts + rng.integers(0, block, size=len(starts)), total - 1)
+
+    # Y and dX: one row in every 128-row block
+    rows = one_per_block(N, 128)
+    nothing = np.zeros((len(rows), 1))
+    Yref, _ = O.forward(X64[rows], W64, None, nothing, want_xproj=False)
+    close(to_np(Y[rows]), Yref, "Y", K["Y"])
+    dXref, _, _, _ = O.backward(dY64[rows], W64, np.zeros((1, Di)), nothing, want_dw=False, want_db=False)
+    close(to_np(dX[rows]), dXref, "dX", K["dX"])
     # db: all of it
-    close(to_np(db), dY64.sum(axis=0), "db")
-    # X_proj: sampled sketch columns j (rows of X_proj), each needs the whole column of S
-    js = sorted(set([0, k - 1] + [int(j) for j in rng.choice(k, size=6, replace=False)]))
-    for j in js:
-        pj = O.generate_p(w.seed, N, k, w.dist, STORE[w.dtype], j, j + 1)[:, 0].astype(np.float64) * c
-        close(to_np(Xp[j]), pj @ X64, f"X_proj[{j}]")
-    # dW: sampled output rows o need G[:, o] = S^T dY[:, o], i.e. all of S once
-    Pm = O.generate_p(w.seed, N, k, w.dist, STORE[w.dtype])          # [N, k] fp32
-    os_ = rng.choice(Do, size=4, replace=False)
-    G = (Pm.astype(np.float64).T @ dY64[:, os_]) * c                   # [k, 4]
+    _, _, dbref, _ = O.backward(dY64, W64[:, :1], np.zeros((1, 1)), np.zeros((N, 1)), want_dx=False, want_dw=False)
+    close(to_np(db)[None, :], dbref[None, :], "db", K["db"])
+    # S once (fp64, scaled): X_proj rows need columns of it, dW rows need all of it
+    S = O.generate_s(w.seed, N, k, w.dist, STORE[w.dtype])
+    js = np.unique(np.concatenate([[0, k - 1], one_per_block(k, 128)]))
+    _, Xpref = O.forward(X64, W64[:1], None, np.ascontiguousarray(S[:, js]), want_y=False)
+    close(to_np(Xp[js]), Xpref, "X_proj", K["X_proj"])
+    # dW: one row in every 128-row block of D_out; stage-wise (the GPU's own X_proj, as rmm_backward receives it)
+    os_ = one_per_block(Do, 128)
     Xp64 = to_np(Xp)
-    for t, o in enumerate(os_):
-        close(to_np(dW[o]), G[:, t] @ Xp64, f"dW[{o}]")
-    # properties that hold at any size: unbiasedness scale -- |dW| is of the order of |dY^T X|
+    _, dWref, _, G = O.backward(np.ascontiguousarray(dY64[:, os_]), W64[os_], Xp64, S, want_dx=False, want_db=False)
+    close(to_np(dW[os_]), dWref, "dW", K["dW"], dw_operand_term(G, Xp64, w.dtype))
     return True
 
 
