@@ -34,7 +34,7 @@ DEFAULT_WORKLOAD = "large_ffn_up_rho0.1"
 # the schedule, not the token count).
 NCU_DRAM_BYTES = {("large_ffn_up_rho0.1", "sdy"): (33.698304e6 / 4096, 14.677504e6)}
 
-STEP_ORDER = ("y", "sketch", "dx", "sdy", "dw", "db")
+STEP_ORDER = ("fwd", "bwd", "y", "sketch", "dx", "sdy", "dw", "db")
 E2E_LANES = 3    # streams (each with its own staging buffers and thread) that take the end-to-end steps in turn
 
 
@@ -259,7 +259,7 @@ def main():
     barrier()
     assert P.rmm_last_device_status(ws) == P.RMM_OK
 
-    launches_per_step = 7
+    launches_before = P.rmm_layer_launch_count()
     P.rmm_profile_enable(min(args.steps, 200) * 6)     # per-kernel events for the first 200 timed steps
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
@@ -272,6 +272,7 @@ def main():
     barrier()
     sampler.stop_flag.set()
     sampler.join()
+    gpu_launches = P.rmm_layer_launch_count() - launches_before     # the library's own count of its kernel launches
     ms_total = e0.elapsed_time(e1)
     assert P.rmm_last_device_status(ws) == P.RMM_OK
     records = P.rmm_profile_read(min(args.steps, 200) * 6)
@@ -289,7 +290,8 @@ def main():
         if v:
             per_kernel[name] = {"ms": float(np.mean(v)), "launches_timed": len(v)}
     peaks = load_peaks()
-    flops_of = {"y": fl["y"], "sketch": fl["sketch"], "dx": fl["dx"], "sdy": fl["sdy"], "dw": fl["dw"]}
+    flops_of = {"y": fl["y"], "sketch": fl["sketch"], "dx": fl["dx"], "sdy": fl["sdy"], "dw": fl["dw"],
+                "fwd": fl["y"] + fl["sketch"], "bwd": fl["dx"] + fl["sdy"]}
     for name, d in per_kernel.items():
         if name in flops_of:
             d["tflops"] = flops_of[name] / (d["ms"] * 1e-3) / 1e12
@@ -387,7 +389,7 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16" if w.dtype == R.DTYPE_BF16 else "f32", "data": "synthetic",
                 "config": workload_config(w), "clocks": clocks, "e2e": e2e,
-                "gpu_launches": launches_per_step * args.steps, "roofline": roofline, "cpu_baseline": cpu,
+                "gpu_launches": gpu_launches, "roofline": roofline, "cpu_baseline": cpu,
                 "pct_of_tensor_peak": {"burst": 100 * value / world / peaks["bf16_tflops"],
                                        "sustained": 100 * value / world / peaks["bf16_tflops_sustained"],
                                        "of": peaks["source"]},

@@ -120,6 +120,21 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj,
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * How the bf16 passes are executed (no counterpart in the paper; process-wide, takes effect for later calls).
+ *   0 (default): the dense product and the sketch of a pass (Y and S^T X; dX and S^T dY) are two persistent
+ *      kernels that run at the same time on disjoint sets of SMs; the sketch kernel is queued on a stream of the
+ *      library's own that forks from and joins the caller's stream through events, so to the caller the pass is
+ *      still ordered on its stream.  The library creates these side streams (eight per device) at its first call
+ *      on a device and keeps them until the process exits.
+ *   1: both parts of a pass in ONE launch (a kernel whose CTA pairs take sketch units and dense tiles from one
+ *      static schedule).  Same results up to the order of the fp32 partial sums; slower on B200 for the Gaussian
+ *      sketch (the generation of S does not keep up with two SMs that share every generated entry through the
+ *      tensor cores' pair mode), kept as an alternative and for measurements.
+ * Returns RMM_ERR_INVALID_ARG for any other value.
+ */
+rmm_status rmm_set_pass_mode(int mode);
+
+/*
  * Writes the sketch matrix itself, S_out [N, B_proj] row-major in the given dtype
  * holding the UNSCALED entries P (multiply by fp32 1/sqrt(B_proj) to get S, Eq. 5).
  * Not part of the layer: it exists so that the generator can be compared bit for bit
@@ -152,6 +167,20 @@ int64_t rmm_debug_sketch_schedule(int64_t rows, int64_t cols, int64_t tokens, in
                                   int64_t* records, int64_t cap, int64_t* info);
 
 /*
+ * Host-only testing aid (no device needed): the static work schedule of one pass launch (Algorithm 1,
+ * FORWARD or BACKWARD without its last product) on `max_pairs` CTA pairs.  The dense part is a
+ * gemm_m x gemm_n result contracted over gemm_k (gemm_m = 0: none), in 256 x 256 tiles; the sketch part a
+ * rows x cols result contracted over `tokens` (rows = 0: none), in tiles of 128 rows x nat x 256 columns cut
+ * along the tokens into nb blocks of blen 64-token steps.  Writes to out (host memory, at most cap values):
+ *   num_pairs, dense tiles, dense column tiles, K blocks, sketch row tiles, column groups, nat,
+ *   64-token steps, nb, blen, then num_pairs + 1 values b[p]: pair p computes the dense tiles
+ *   [b[p], b[p + 1]).  Sketch unit i = block * (row tiles * groups) + tile goes to pair i % num_pairs.
+ * Returns the number of values that exist, or -1 for invalid arguments.
+ */
+int64_t rmm_debug_pass_schedule(int64_t gemm_m, int64_t gemm_n, int64_t gemm_k, int64_t rows, int64_t cols,
+                                int64_t tokens, int max_pairs, int64_t* out, int64_t cap);
+
+/*
  * Reads the status word that the kernels of the last call using this workspace left
  * there.  HOST-synchronous on the device-to-host copy of one word: the caller must
  * have synchronised the stream first.  Returns RMM_OK or RMM_ERR_TIMEOUT (or
@@ -179,9 +208,14 @@ typedef enum {
   RMM_STEP_DX = 2,      /* dX = dY W                (Eq. 2) */
   RMM_STEP_SDY = 3,     /* G = S^T dY               (Algorithm 1, inner product of Eq. 4) */
   RMM_STEP_DW = 4,      /* dW = G^T X_proj          (Eq. 4) */
-  RMM_STEP_DB = 5       /* db = dY^T 1              (Eq. 3), partial sums and final sum */
+  RMM_STEP_DB = 5,      /* db = dY^T 1              (Eq. 3), partial sums and final sum */
+  RMM_STEP_FWD = 6,     /* Y and X_proj in one launch       (Algorithm 1, FORWARD) */
+  RMM_STEP_BWD = 7      /* dX, G = S^T dY and db in one launch (Algorithm 1, BACKWARD, all but the last product) */
 } rmm_step;
 rmm_status rmm_profile_enable(int capacity);
+/* Number of kernels that rmm_forward / rmm_backward (and their host-buffer forms) have launched in this
+ * process so far (no counterpart in the paper; a benchmark's launch count). */
+int64_t rmm_layer_launch_count(void);
 int rmm_profile_read(int* step_ids, float* milliseconds, int max_records);
 
 /*

@@ -20,9 +20,9 @@ EXPORTS = ("rmm_workspace_bytes", "rmm_forward", "rmm_backward", "rmm_debug_gene
            "rmm_last_device_status", "rmm_status_string", "rmm_host_staging_bytes",
            "rmm_forward_host", "rmm_backward_host", "rmm_profile_enable", "rmm_profile_read",
            "rmm_bias_grad_static", "rmm_debug_gauss_words", "rmm_debug_sketch_schedule",
-           "rmm_variance_probe_workspace_bytes", "rmm_variance_probe")
+           "rmm_variance_probe_workspace_bytes", "rmm_variance_probe", "rmm_debug_pass_schedule", "rmm_layer_launch_count", "rmm_set_pass_mode")
 RMM_BIAS_GRAD_STATIC_MAX_D_OUT = 4096
-STEP_NAMES = ("y", "sketch", "dx", "sdy", "dw", "db")
+STEP_NAMES = ("y", "sketch", "dx", "sdy", "dw", "db", "fwd", "bwd")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2201_13195_b200.build` "
@@ -54,10 +54,16 @@ _lib.rmm_debug_gauss_words.argtypes = [_vp, _i64, _vp, _vp]
 _lib.rmm_debug_gauss_words.restype = _int
 _lib.rmm_debug_sketch_schedule.argtypes = [_i64, _i64, _i64, _int, _int, _vp, _i64, _vp]
 _lib.rmm_debug_sketch_schedule.restype = _i64
+_lib.rmm_debug_pass_schedule.argtypes = [_i64, _i64, _i64, _i64, _i64, _i64, _int, _vp, _i64]
+_lib.rmm_debug_pass_schedule.restype = _i64
 _lib.rmm_variance_probe_workspace_bytes.argtypes = [_i64, _i64, _i64]
 _lib.rmm_variance_probe_workspace_bytes.restype = _sz
 _lib.rmm_variance_probe.argtypes = [_vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _vp, _vp, _vp, _sz, _vp]
 _lib.rmm_variance_probe.restype = _int
+_lib.rmm_set_pass_mode.argtypes = [_int]
+_lib.rmm_set_pass_mode.restype = _int
+_lib.rmm_layer_launch_count.argtypes = []
+_lib.rmm_layer_launch_count.restype = _i64
 _lib.rmm_profile_enable.argtypes = [_int]
 _lib.rmm_profile_enable.restype = _int
 _lib.rmm_profile_read.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_float), _int]
@@ -241,6 +247,30 @@ def rmm_debug_gauss_words(words, stream=None):
     _check(_lib.rmm_debug_gauss_words(_ptr(words), words.numel(), _ptr(out), _stream_ptr(stream)),
            "rmm_debug_gauss_words")
     return out
+
+
+def rmm_set_pass_mode(mode: int) -> None:
+    """0: the two kernels of a pass side by side (default); 1: one launch per pass."""
+    _check(_lib.rmm_set_pass_mode(int(mode)), "rmm_set_pass_mode")
+
+
+def rmm_layer_launch_count() -> int:
+    return int(_lib.rmm_layer_launch_count())
+
+
+def rmm_debug_pass_schedule(gemm, sketch, max_pairs=74):
+    """The static schedule of one pass launch (host only).  gemm = (M, N, K) or None, sketch = (rows, cols, tokens) or None."""
+    gm, gn, gk = gemm if gemm else (0, 0, 0)
+    rows, cols, tokens = sketch if sketch else (0, 0, 0)
+    n = _lib.rmm_debug_pass_schedule(gm, gn, gk, rows, cols, tokens, max_pairs, None, 0)
+    if n < 0:
+        raise ValueError("invalid arguments")
+    buf = (C.c_int64 * n)()
+    _lib.rmm_debug_pass_schedule(gm, gn, gk, rows, cols, tokens, max_pairs, C.addressof(buf), n)
+    names = ("num_pairs", "gemm_tiles", "tiles_n", "num_kb", "tiles_m", "groups", "nat", "ksteps", "nb", "blen")
+    d = {k: int(buf[i]) for i, k in enumerate(names)}
+    d["gemm_begin"] = [int(buf[10 + i]) for i in range(d["num_pairs"] + 1)]
+    return d
 
 
 def rmm_debug_sketch_schedule(rows, cols, tokens, max_ctas=148, mode=0):

@@ -28,6 +28,16 @@ def nvcc_command(out: str, extra=()):
             *[os.path.join(CSRC, s) for s in SOURCES], *extra]
 
 
+def build_trace(out: str) -> str:
+    """A second library with the pass kernel's cycle accounting compiled in (-DRMM_PASS_TRACE): for profiling
+    sessions only, never loaded by the package."""
+    res = subprocess.run(nvcc_command(out, ["-DRMM_PASS_TRACE"]), capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed building the trace library")
+    return out
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source_mtime():
         return LIB
@@ -42,4 +52,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    if "--trace" in sys.argv:
+        print(build_trace(sys.argv[sys.argv.index("--trace") + 1]))
+    else:
+        print(build(force=True, verbose="-v" in sys.argv))

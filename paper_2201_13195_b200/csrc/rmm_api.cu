@@ -6,6 +6,9 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+#include <chrono>
+#include <cstring>
 #include <mutex>
 #include <vector>
 
@@ -14,6 +17,7 @@
 #include "tc_gemm.cuh"
 #include "fwht_kernels.cuh"
 #include "tc_sketch.cuh"
+#include "tc_pass.cuh"
 #include "variance_kernels.cuh"
 
 namespace {
@@ -28,15 +32,52 @@ inline size_t elem_bytes(rmm_dtype dt) { return dt == RMM_DTYPE_BF16 ? 2 : 4; }
 // [status word | G = S^T dY | scratch], scratch = fp32 partial tiles of the sketch kernels
 // (bf16 mode) or partial column sums of db (fp32 mode).
 struct Workspace {
-  size_t status_off, g_off, scratch_off, total;
+  size_t status_off, ticket_off, g_off, scratch_off, total;
   int db_rows_per_slice, db_slices;
 };
+
+// Geometry of the sketch part of a pass (tc_pass.cuh): a pair tile is 128 sketch rows x nat x 256 data
+// columns; the column groups are balanced so that no group is mostly padding.
+struct SketchGeometry {
+  int tiles_m, groups, nat, ksteps;
+  int tiles() const { return tiles_m * groups; }
+  // Upper bound of the number of token blocks per tile, whatever the device: at most kMaxUnits units in all
+  // (one or two per CTA pair of the largest grid) unless the tiles alone are more.
+  static constexpr int kMaxUnits = 2 * tc::PS_MAX_PAIRS;
+  int nb_cap() const {
+    int c = kMaxUnits / tiles();
+    if (c < 1) c = 1;
+    return c < ksteps ? c : ksteps;
+  }
+  size_t scratch_bytes() const {
+    return (size_t)tiles() * (size_t)nb_cap() * tc::PS_ROWS * (size_t)nat * 256 * sizeof(float);
+  }
+};
+
+SketchGeometry sketch_geometry(int64_t rows, int64_t cols, int64_t tokens) {
+  SketchGeometry g;
+  const int64_t t256 = (cols + 255) / 256;
+  g.groups = (int)((t256 + tc::PS_MAX_NAT - 1) / tc::PS_MAX_NAT);
+  g.nat = (int)((t256 + g.groups - 1) / g.groups);
+  g.tiles_m = (int)((rows + tc::PS_ROWS - 1) / tc::PS_ROWS);
+  g.ksteps = (int)((tokens + 63) / 64);
+  return g;
+}
 
 Workspace workspace_layout(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rmm_dtype dt) {
   Workspace w;
   w.status_off = 0;
-  w.g_off = kAlign;
-  size_t off = w.g_off + align_up((size_t)k * (size_t)D_out * elem_bytes(dt));
+  w.ticket_off = kAlign;
+  size_t off = w.ticket_off;
+  size_t scratch_pass = 0;
+  if (dt == RMM_DTYPE_BF16) {
+    const SketchGeometry gf = sketch_geometry(k, D_in, N), gb = sketch_geometry(k + 1, D_out, N);
+    const int tmax = gf.tiles() > gb.tiles() ? gf.tiles() : gb.tiles();
+    off += align_up((size_t)tmax * sizeof(unsigned long long));
+    scratch_pass = gf.scratch_bytes() > gb.scratch_bytes() ? gf.scratch_bytes() : gb.scratch_bytes();
+  }
+  w.g_off = off;
+  off = w.g_off + align_up((size_t)k * (size_t)D_out * elem_bytes(dt));
   int64_t rps = 256;
   if ((N + rps - 1) / rps > 256) rps = (N + 255) / 256;
   w.db_rows_per_slice = (int)rps;
@@ -48,6 +89,7 @@ Workspace workspace_layout(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rm
     const long long tf = ((k + tc::SK_BM - 1) / tc::SK_BM) * ((D_in + tc::SK_BN - 1) / tc::SK_BN);
     const long long tb = ((k + 1 + tc::SK_BM - 1) / tc::SK_BM) * ((D_out + tc::SK_BN - 1) / tc::SK_BN);
     scratch = (size_t)((tf > tb ? tf : tb) + tc::SK_MAX_CTAS) * tc::SK_TILE_ELEMS * sizeof(float);
+    if (scratch_pass > scratch) scratch = scratch_pass;
   }
   off += align_up(scratch);
   w.total = off;
@@ -65,6 +107,14 @@ struct DeviceState {
   int num_sms = 0;
   int gemm_pairs = 0;                         // CTA pairs of the GEMM kernel resident at once
   int sketch_clusters[5] = {0, 0, 0, 0, 0};   // [C]: clusters of C CTAs of the sketch kernel resident at once
+  int pass_pairs = 0;                         // CTA pairs of the pass kernel resident at once
+  // side lanes for the two kernels of a pass that run at the same time: a stream and two events each
+  static constexpr int kLanes = 8;
+  cudaStream_t lane_stream[kLanes] = {};
+  cudaEvent_t lane_fork[kLanes] = {}, lane_join[kLanes] = {};
+  std::mutex lane_mutex[kLanes];
+  std::atomic<unsigned> next_lane{0};
+  bool lanes_ok = false;
 };
 
 template <typename K>
@@ -79,6 +129,17 @@ SketchKernelFn sketch_kernel_fn(int c, int dist) {
       {tc::sketch_kernel<1, 0>, tc::sketch_kernel<1, 1>, tc::sketch_kernel<1, 2>, tc::sketch_kernel<1, 3>},
       {tc::sketch_kernel<2, 0>, tc::sketch_kernel<2, 1>, tc::sketch_kernel<2, 2>, tc::sketch_kernel<2, 3>}};
   return table[c == 2 ? 1 : 0][dist & 3];
+}
+
+// The pass kernel for an operand mode of the dense part (B_K: Y = X W^T, B_MN: dX = dY W) and a distribution.
+typedef void (*PassKernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, tc::PassParams,
+                             PhiloxKey);
+PassKernelFn pass_kernel_fn(int bmode, int dist) {
+  static const PassKernelFn table[2][4] = {
+      {tc::pass_kernel<tc::B_K, 0>, tc::pass_kernel<tc::B_K, 1>, tc::pass_kernel<tc::B_K, 2>, tc::pass_kernel<tc::B_K, 3>},
+      {tc::pass_kernel<tc::B_MN, 0>, tc::pass_kernel<tc::B_MN, 1>, tc::pass_kernel<tc::B_MN, 2>,
+       tc::pass_kernel<tc::B_MN, 3>}};
+  return table[bmode == tc::B_MN ? 1 : 0][dist & 3];
 }
 
 // How many clusters of `c` CTAs of kernel `k` can be resident on the device at once.
@@ -121,10 +182,23 @@ void init_device_state(DeviceState& st, int dev) {
   a &= allow_big_smem(tc::gemm_kernel<tc::A_MN, tc::B_MN>, tc::GEMM_SMEM_BYTES);
   for (int c = 1; c <= 2; ++c)
     for (int d = 0; d < 4; ++d) a &= allow_big_smem(sketch_kernel_fn(c, d), tc::SK_SMEM_BYTES);
+  for (int bm = 0; bm < 2; ++bm)
+    for (int d = 0; d < 4; ++d) a &= allow_big_smem(pass_kernel_fn(bm, d), tc::PS_SMEM_BYTES);
   if (a) {
+    a &= query_clusters(tc::pass_kernel<tc::B_K, 0>, 2, &st.pass_pairs, tc::PS_THREADS, tc::PS_SMEM_BYTES);
+    if (st.pass_pairs > tc::PS_MAX_PAIRS) st.pass_pairs = tc::PS_MAX_PAIRS;
     st.sketch_clusters[1] = st.num_sms < tc::SK_MAX_CTAS ? st.num_sms : tc::SK_MAX_CTAS;
     a &= query_clusters(tc::sketch_kernel<2, 0>, 2, &st.sketch_clusters[2]);   // the same for every distribution
     a &= query_clusters(tc::gemm_kernel<tc::A_K, tc::B_K>, 2, &st.gemm_pairs, 64 + 32 * tc::NEPI, tc::GEMM_SMEM_BYTES);
+  }
+  if (a) {
+    bool l = true;
+    for (int i = 0; i < DeviceState::kLanes && l; ++i) {
+      l &= cudaStreamCreateWithFlags(&st.lane_stream[i], cudaStreamNonBlocking) == cudaSuccess;
+      l &= cudaEventCreateWithFlags(&st.lane_fork[i], cudaEventDisableTiming) == cudaSuccess;
+      l &= cudaEventCreateWithFlags(&st.lane_join[i], cudaEventDisableTiming) == cudaSuccess;
+    }
+    st.lanes_ok = l;
   }
   st.ok = a;
 }
@@ -172,6 +246,10 @@ bool make_tmap_slabs(CUtensorMap* map, const void* base, int64_t rows, int64_t c
                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Kernels launched by rmm_forward / rmm_backward (and their host-buffer wrappers) since the library was loaded.
+std::atomic<long long> g_layer_launches{0};
+inline void note_launches(int n) { g_layer_launches.fetch_add(n, std::memory_order_relaxed); }
+
 // ------------------------------------------------------------------ per-kernel timing (benchmarks)
 struct ProfileRecord { int step; cudaEvent_t t0, t1; };
 struct Profiler {
@@ -212,7 +290,8 @@ int tc_grid_ctas(int64_t M, int64_t N) {
 
 template <int AMODE, int BMODE>
 rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, int64_t M, int64_t N, int64_t K,
-                     float alpha, int* status, cudaStream_t stream, double* sumsq = nullptr, bool clear_status = false) {
+                     float alpha, int* status, cudaStream_t stream, double* sumsq = nullptr, bool clear_status = false,
+                     int pairs_limit = 0) {
   CUtensorMap tmA, tmB, tmC;
   bool ok = make_tmap(&tmC, c, M, N, 32);        // store boxes of the epilogue: [32 rows][64 columns]
   if (AMODE == tc::A_K) ok &= make_tmap(&tmA, a, M, K, tc::BM);
@@ -224,7 +303,8 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   p.M = M; p.N = N; p.K = K;
   p.bias = bias; p.alpha = alpha; p.status = status; p.sumsq = sumsq; p.clear_status = clear_status ? 1 : 0;
   const int64_t tiles = ((N + tc::BN - 1) / tc::BN) * ((M + tc::PAIR_M - 1) / tc::PAIR_M);
-  const int max_pairs = device_state().gemm_pairs;
+  int max_pairs = device_state().gemm_pairs;
+  if (pairs_limit > 0 && pairs_limit < max_pairs) max_pairs = pairs_limit;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -236,6 +316,7 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (cudaLaunchKernelEx(&cfg, tc::gemm_kernel<AMODE, BMODE>, tmA, tmB, tmC, p) != cudaSuccess) return RMM_ERR_CUDA;
+  note_launches(1);
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
 
@@ -245,34 +326,59 @@ rmm_status launch_tc(const void* a, const void* b, void* c, const void* bias, in
 // RMM_ERR_UNSUPPORTED when the shape is outside the fast path (the caller then takes the dense kernel).
 // scratch holds, in this order: the grouped column list, the per-block column sums, the stage-1 result
 // T for as many columns per round as fit.
-rmm_status launch_sors_fast(const void* b, void* out, void* ones_out, int64_t k, int64_t cols, int64_t tokens, float c,
-                            const PhiloxKey& pk, void* scratch, size_t scratch_bytes, int* status, cudaStream_t stream,
-                            bool clear_status) {
+// Layout of the fast path's scratch for a sketch of k rows over `cols` columns and `tokens` rows; false when the
+// shape is outside the fast path (Hadamard order below 128 or above 16384, or scratch too small).
+struct SorsFastPlan {
+  uint32_t mask;
+  int A;
+  size_t entries_off, colsum_off, t_off;
+  int64_t wslab;
+};
+bool sors_fast_plan(int64_t k, int64_t cols, int64_t tokens, size_t scratch_bytes, SorsFastPlan* plan) {
   const uint32_t mask = sors_mask_for(tokens);
   const int64_t L = (int64_t)mask + 1;
-  if (L < FW_ROWS || L > (int64_t)FW_ROWS * FW_ROWS) return RMM_ERR_UNSUPPORTED;
+  if (L < FW_ROWS || L > (int64_t)FW_ROWS * FW_ROWS) return false;
   const int A = (int)(L / FW_ROWS);
-  uint8_t* base = reinterpret_cast<uint8_t*>(scratch);
-  size_t off = 0;
-  SorsGroups g;
-  g.offsets = reinterpret_cast<int*>(base + off);
-  off += align_up(129 * sizeof(int));
-  g.entries = reinterpret_cast<int2*>(base + off);
+  size_t off = align_up(129 * sizeof(int));
+  const size_t entries_off = off;
   off += align_up((size_t)k * sizeof(int2));
-  if (off + 2 * kAlign >= scratch_bytes) return RMM_ERR_UNSUPPORTED;
+  if (off + 2 * kAlign >= scratch_bytes) return false;
   const size_t per_col = (size_t)A * sizeof(float) + (size_t)L * 2;       // column sums + T, per column of a round
   const int64_t cols64 = (cols + FW_COLS - 1) / FW_COLS * FW_COLS;
   int64_t wslab = (int64_t)((scratch_bytes - off - 2 * kAlign) / per_col) / FW_COLS * FW_COLS;
   if (wslab > cols64) wslab = cols64;
-  if (wslab < FW_COLS) return RMM_ERR_UNSUPPORTED;
+  if (wslab < FW_COLS) return false;
   {   // rounds of equal width rather than full ones and a narrow last one
     const int64_t rounds = (cols64 + wslab - 1) / wslab;
     wslab = ((cols64 + rounds - 1) / rounds + FW_COLS - 1) / FW_COLS * FW_COLS;
   }
-  float* colsum = reinterpret_cast<float*>(base + off);
-  off += align_up((size_t)A * (size_t)wslab * sizeof(float));
-  __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(base + off);
+  if (plan) {
+    plan->mask = mask; plan->A = A; plan->entries_off = entries_off; plan->colsum_off = off;
+    plan->t_off = off + align_up((size_t)A * (size_t)wslab * sizeof(float));
+    plan->wslab = wslab;
+  }
+  return true;
+}
+bool sors_fast_supported(int64_t k, int64_t cols, int64_t tokens, size_t scratch_bytes) {
+  return sors_fast_plan(k, cols, tokens, scratch_bytes, nullptr);
+}
+
+rmm_status launch_sors_fast(const void* b, void* out, void* ones_out, int64_t k, int64_t cols, int64_t tokens, float c,
+                            const PhiloxKey& pk, void* scratch, size_t scratch_bytes, int* status, cudaStream_t stream,
+                            bool clear_status) {
+  SorsFastPlan plan;
+  if (!sors_fast_plan(k, cols, tokens, scratch_bytes, &plan)) return RMM_ERR_UNSUPPORTED;
+  const uint32_t mask = plan.mask;
+  const int A = plan.A;
+  const int64_t wslab = plan.wslab;
+  uint8_t* base = reinterpret_cast<uint8_t*>(scratch);
+  SorsGroups g;
+  g.offsets = reinterpret_cast<int*>(base);
+  g.entries = reinterpret_cast<int2*>(base + plan.entries_off);
+  float* colsum = reinterpret_cast<float*>(base + plan.colsum_off);
+  __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(base + plan.t_off);
   sors_group_kernel<<<1, 1024, 0, stream>>>(pk, k, mask, g, status, clear_status ? 1 : 0);
+  note_launches(1);
   if (cudaGetLastError() != cudaSuccess) return RMM_ERR_CUDA;
   const __nv_bfloat16* B = reinterpret_cast<const __nv_bfloat16*>(b);
   __nv_bfloat16* O = reinterpret_cast<__nv_bfloat16*>(out);
@@ -283,6 +389,7 @@ rmm_status launch_sors_fast(const void* b, void* out, void* ones_out, int64_t k,
     fwht_stage1_kernel<<<dim3(slabs, (unsigned)A), FW_THREADS, 0, stream>>>(B + c0, cols, tokens, width, pk, T, wslab,
                                                                            ones ? colsum : nullptr);
     if (cudaGetLastError() != cudaSuccess) return RMM_ERR_CUDA;
+    note_launches(2);
     fwht_stage2_kernel<<<dim3(slabs, FW_ROWS), FW_THREADS, 0, stream>>>(T, wslab, A, width, g, c, O + c0, cols,
                                                                        ones ? colsum : nullptr, ones ? ones + c0 : nullptr);
     if (cudaGetLastError() != cudaSuccess) return RMM_ERR_CUDA;
@@ -292,12 +399,7 @@ rmm_status launch_sors_fast(const void* b, void* out, void* ones_out, int64_t k,
 
 rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, int64_t cols, int64_t tokens, float c,
                          int dist, const PhiloxKey& pk, float* partial, int* status, cudaStream_t stream,
-                         bool clear_status = false, size_t scratch_bytes = 0) {
-  if (dist == RMM_DIST_SORS_HADAMARD && scratch_bytes > 0) {
-    const rmm_status fs = launch_sors_fast(b, out, ones_out, k, cols, tokens, c, pk, partial, scratch_bytes, status, stream,
-                                           clear_status);
-    if (fs != RMM_ERR_UNSUPPORTED) return fs;
-  }
+                         bool clear_status = false, int clusters_limit = 0) {
   CUtensorMap tmB;
   const bool slab_map = cols % 64 == 0;
   if (!(slab_map ? make_tmap_slabs(&tmB, b, tokens, cols, tc::SK_BK, tc::SK_BN / 64)
@@ -316,7 +418,9 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   p.status = status;
   p.clear_status = clear_status ? 1 : 0;
   const int C = tc::sketch_cluster_size(cols);
-  p.sched = tc::make_sketch_schedule(p.rows, cols, tokens, C, device_state().sketch_clusters[C]);
+  int max_clusters = device_state().sketch_clusters[C];
+  if (clusters_limit > 0 && clusters_limit < max_clusters) max_clusters = clusters_limit;
+  p.sched = tc::make_sketch_schedule(p.rows, cols, tokens, C, max_clusters);
   const int per_tile = C;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
@@ -330,9 +434,173 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   cfg.numAttrs = 1;
   cudaError_t le = cudaLaunchKernelEx(&cfg, sketch_kernel_fn(C, dist), tmB, p, pk);
   if (le != cudaSuccess) return RMM_ERR_CUDA;
+  note_launches(2);
   dim3 rgrid((unsigned)(p.sched.tiles() * per_tile), tc::SK_BN / tc::SKR_CHUNK);
   tc::sketch_reduce_kernel<<<rgrid, tc::SK_BM, 0, stream>>>(p, c, reinterpret_cast<__nv_bfloat16*>(out),
                                                       reinterpret_cast<__nv_bfloat16*>(ones_out));
+  return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------ one pass as one launch (tc_pass.cuh)
+// Static schedule of a pass on `max_pairs` CTA pairs.  The sketch tiles are cut along the tokens into nb
+// blocks each (unit = block * tiles + tile, dealt round-robin: the pairs that run at the same time walk the
+// same token range); the dense tiles then go, one by one, to the pair that is least loaded.  nb is the
+// candidate with the smallest estimated makespan, in units of tensor-pipe cycles of a pair.
+tc::PassSchedule make_pass_schedule(bool with_gemm, int64_t gM, int64_t gN, int64_t gK, bool with_sketch, int64_t rows,
+                                    int64_t cols, int64_t tokens, int max_pairs) {
+  tc::PassSchedule s = {};
+  if (max_pairs > tc::PS_MAX_PAIRS) max_pairs = tc::PS_MAX_PAIRS;
+  if (max_pairs < 1) max_pairs = 1;
+  s.tiles_n = 1; s.num_kb = 0; s.gemm_tiles = 0;
+  if (with_gemm) {
+    s.tiles_n = (int)((gN + tc::BN - 1) / tc::BN);
+    s.gemm_tiles = (int)((gM + tc::PAIR_M - 1) / tc::PAIR_M) * s.tiles_n;
+    s.num_kb = (int)((gK + tc::BK - 1) / tc::BK);
+  }
+  s.tiles_m = 0; s.groups = 1; s.nat = 1; s.ksteps = 0; s.nb = 1; s.blen = 1;
+  SketchGeometry g = {};
+  if (with_sketch) {
+    g = sketch_geometry(rows, cols, tokens);
+    s.tiles_m = g.tiles_m; s.groups = g.groups; s.nat = g.nat; s.ksteps = g.ksteps;
+  }
+  const int G = s.gemm_tiles, T = with_sketch ? g.tiles() : 0;
+  // estimated costs (cycles of the pair's tensor pipe): a dense tile, a 64-token sketch step, the drain of a unit
+  const long long cg = (long long)s.num_kb * 512 + 1500;
+  const long long cs = (long long)s.nat * 256 + 64;
+  const long long co = 3500;
+  constexpr int kGreedyMax = 16384;
+  int best_nb = 1, best_pairs = 1;
+  long long best_cost = -1;
+  std::vector<long long> load;
+  const int nb_cap = with_sketch ? g.nb_cap() : 1;
+  for (int nb_try = 1; nb_try <= nb_cap; ++nb_try) {
+    int blen = 1, nb = 1;
+    if (with_sketch) {
+      blen = (s.ksteps + nb_try - 1) / nb_try;
+      nb = (s.ksteps + blen - 1) / blen;
+      if (nb != nb_try) continue;               // the same cut as a smaller candidate
+      if (blen < 4 && nb > 1) break;            // no slivers
+    }
+    const long long units = (long long)T * nb;
+    const int pairs = (int)(units + G < max_pairs ? (units + G > 0 ? units + G : 1) : max_pairs);
+    load.assign((size_t)pairs, 0);
+    for (long long u = 0; u < units; ++u) {
+      const int b = (int)(u / T);
+      const int len = (b + 1) * blen <= s.ksteps ? blen : s.ksteps - b * blen;
+      load[(size_t)(u % pairs)] += (long long)len * cs + co;
+    }
+    for (int t = 0; t < G && G <= kGreedyMax; ++t) {
+      size_t m = 0;
+      for (size_t q = 1; q < load.size(); ++q)
+        if (load[q] < load[m]) m = q;
+      load[m] += cg;
+    }
+    if (G > kGreedyMax)                         // very many dense tiles: the sketch units no longer matter for the balance
+      for (long long& v : load) v += (long long)((G + pairs - 1) / pairs) * cg;
+    long long cost = 0;
+    for (long long v : load) cost = v > cost ? v : cost;
+    cost += (long long)nb * 40;                 // more blocks: more partial tiles to add up
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost; best_nb = nb; best_pairs = pairs;
+    }
+    if (!with_sketch) break;
+  }
+  s.nb = best_nb;
+  s.blen = with_sketch ? (s.ksteps + best_nb - 1) / best_nb : 1;
+  s.num_pairs = best_pairs;
+  // dense tiles: counts by the same greedy rule, then consecutive ranges
+  std::vector<int> count((size_t)best_pairs, 0);
+  load.assign((size_t)best_pairs, 0);
+  const long long units = (long long)T * s.nb;
+  for (long long u = 0; u < units; ++u) {
+    const int b = (int)(u / T);
+    const int len = (b + 1) * s.blen <= s.ksteps ? s.blen : s.ksteps - b * s.blen;
+    load[(size_t)(u % best_pairs)] += (long long)len * cs + co;
+  }
+  for (int t = 0; t < G && G <= kGreedyMax; ++t) {
+    size_t m = 0;
+    for (size_t q = 1; q < load.size(); ++q)
+      if (load[q] < load[m]) m = q;
+    load[m] += cg;
+    ++count[m];
+  }
+  if (G > kGreedyMax)
+    for (int q = 0; q < best_pairs; ++q) count[(size_t)q] = G / best_pairs + (q < G % best_pairs ? 1 : 0);
+  int acc = 0;
+  for (int q = 0; q <= tc::PS_MAX_PAIRS; ++q) {
+    s.gemm_begin[q] = acc;
+    if (q < best_pairs) acc += count[(size_t)q];
+  }
+  s.gemm_begin[tc::PS_MAX_PAIRS + 1] = acc;
+  return s;
+}
+
+// 48-bit tag of a launch: the tickets of the sketch tiles carry it, so that counts left in a workspace by
+// earlier launches (or never initialised) read as zero.
+unsigned long long next_launch_tag() {
+  static std::atomic<unsigned long long> counter{
+      (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count() * 0x9E3779B97F4A7C15ull};
+  return (counter.fetch_add(1) + 1) & ((1ull << 48) - 1);
+}
+
+// One pass: optional dense part C = A B^T (+ bias), A [M][K]; B [N][K] (B_K) or [K][N] (B_MN); optional sketch
+// part out[j][d] = c sum_n P[n][j] data[n][d] (+ ones_out[d] = sum_n data[n][d]).
+struct PassArgs {
+  // dense
+  const void *a = nullptr, *b = nullptr, *bias = nullptr;
+  void* c = nullptr;
+  int64_t M = 0, N = 0, K = 0;
+  int bmode = tc::B_K;
+  // sketch
+  const void* data = nullptr;
+  void *out = nullptr, *ones_out = nullptr;
+  int64_t k = 0, cols = 0, tokens = 0;
+  float scale = 1.0f;
+  int dist = 0;
+};
+
+rmm_status launch_pass(const PassArgs& a, const PhiloxKey& pk, float* partial, unsigned long long* tickets, int* status,
+                       cudaStream_t stream, bool clear_status) {
+  const bool with_gemm = a.c != nullptr, with_sketch = a.out != nullptr;
+  if (!with_gemm && !with_sketch) return RMM_OK;
+  const int64_t rows = a.k + (a.ones_out ? 1 : 0);
+  tc::PassParams p = {};
+  p.sched = make_pass_schedule(with_gemm, a.M, a.N, a.K, with_sketch, rows, a.cols, a.tokens, device_state().pass_pairs);
+  CUtensorMap tmA, tmB, tmC, tmD;
+  memset(&tmA, 0, sizeof(tmA)); memset(&tmB, 0, sizeof(tmB)); memset(&tmC, 0, sizeof(tmC)); memset(&tmD, 0, sizeof(tmD));
+  bool ok = true;
+  if (with_gemm) {
+    ok &= make_tmap(&tmC, a.c, a.M, a.N, 32);
+    ok &= make_tmap(&tmA, a.a, a.M, a.K, tc::BM);
+    if (a.bmode == tc::B_K) ok &= make_tmap(&tmB, a.b, a.N, a.K, tc::BN_HALF);
+    else ok &= make_tmap(&tmB, a.b, a.K, a.N, tc::BK);
+  }
+  const bool slab_map = a.cols % 64 == 0;
+  if (with_sketch)
+    ok &= slab_map ? make_tmap_slabs(&tmD, a.data, a.tokens, a.cols, 32, 2 * p.sched.nat)
+                   : make_tmap(&tmD, a.data, a.tokens, a.cols, 32);
+  if (!ok) return RMM_ERR_CUDA;
+  p.M = a.M; p.N = a.N; p.K = a.K; p.bias = a.bias;
+  p.rows = rows; p.b_proj = a.k; p.cols = a.cols; p.tokens = a.tokens;
+  p.scale = a.scale; p.ones_row = a.ones_out ? 1 : 0; p.slab_map = slab_map ? 1 : 0;
+  p.sors_mask = sors_mask_for(a.tokens > 0 ? a.tokens : 1);
+  p.partial = partial; p.tickets = tickets; p.tag = next_launch_tag();
+  p.sk_out = reinterpret_cast<__nv_bfloat16*>(a.out);
+  p.ones_out = reinterpret_cast<__nv_bfloat16*>(a.ones_out);
+  p.status = status; p.clear_status = clear_status ? 1 : 0;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(2 * (unsigned)p.sched.num_pairs);
+  cfg.blockDim = dim3(tc::PS_THREADS);
+  cfg.dynamicSmemBytes = tc::PS_SMEM_BYTES;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, pass_kernel_fn(a.bmode, a.dist), tmA, tmB, tmC, tmD, p, pk) != cudaSuccess)
+    return RMM_ERR_CUDA;
+  note_launches(1);
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
 
@@ -340,6 +608,7 @@ template <typename T, bool GEN_A>
 rmm_status launch_simt(const SimtGemmArgs& g, const PhiloxKey& pk, cudaStream_t stream) {
   dim3 grid((unsigned)((g.N + SIMT_BN - 1) / SIMT_BN), (unsigned)((g.M + SIMT_BM - 1) / SIMT_BM));
   simt_gemm_kernel<T, GEN_A><<<grid, SIMT_THREADS, 0, stream>>>(g, pk);
+  note_launches(1);
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
 
@@ -360,11 +629,72 @@ rmm_status launch_db(const void* dY, int64_t N, int64_t D_out, const Workspace& 
                      cudaStream_t stream) {
   float* partial = reinterpret_cast<float*>(ws + w.scratch_off);
   dim3 grid((unsigned)((D_out + 255) / 256), (unsigned)w.db_slices);
+  note_launches(2);
   db_partial_kernel<T><<<grid, 256, 0, stream>>>(reinterpret_cast<const T*>(dY), N, D_out, w.db_rows_per_slice, partial);
   db_finish_kernel<T><<<(unsigned)((D_out + 255) / 256), 256, 0, stream>>>(partial, w.db_slices, D_out,
                                                                            reinterpret_cast<T*>(db));
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
+
+// ------------------------------------------------------------------ a pass as two kernels that run at the same time
+// The dense product and the sketch of a pass (Algorithm 1: Y and S^T X; dX and S^T dY) read the same token-sized
+// operand and do not depend on each other.  Each is a persistent kernel whose static schedule is built for the
+// number of CTA pairs / clusters it is given, so the two can share the GPU: the dense kernel gets `pairs` CTA
+// pairs on the caller's stream, the sketch kernel the remaining clusters on a side stream that forks from and
+// joins the caller's stream through events.  Short tails of one kernel are filled by the other, the fixed costs of
+// the launches overlap, and the shared operand is in L2 for whichever reads it second.  If the device cannot hold
+// both grids at once (other work running) the kernels simply run one after the other: neither waits for the other.
+struct PassSplit {
+  int gemm_pairs;       // 0: no split, both kernels get the whole device one after the other
+  int sketch_clusters;
+};
+
+PassSplit plan_pass_split(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens) {
+  PassSplit best = {0, 0};
+  const DeviceState& ds = device_state();
+  const int C = tc::sketch_cluster_size(cols);
+  const int total = ds.gemm_pairs < ds.sketch_clusters[2] ? ds.gemm_pairs : ds.sketch_clusters[2];   // SM pairs
+  if (total < 2 || !ds.lanes_ok) return best;
+  const long long G = ((gN + tc::BN - 1) / tc::BN) * ((gM + tc::PAIR_M - 1) / tc::PAIR_M);
+  const long long num_kb = (gK + tc::BK - 1) / tc::BK;
+  // costs in SM cycles: a dense tile (4 MMAs of 128 cycles per K block, plus fill and epilogue), a 64-token sketch step
+  const long long cg = num_kb * 540 + 3000, cstep = 1460, fixed = 6000;
+  auto gemm_cost = [&](int pairs) { return ((G + pairs - 1) / pairs) * cg + fixed; };
+  auto sketch_cost = [&](int clusters) {
+    const tc::SketchSchedule sc = tc::make_sketch_schedule(rows, cols, tokens, C, C == 2 ? clusters : 2 * clusters);
+    return sc.est_steps * cstep + fixed + 9000;    // + the reduction kernel
+  };
+  const long long serial = gemm_cost(total) + sketch_cost(total);
+  long long best_cost = serial;
+  for (int pg = 1; pg < total; ++pg) {
+    const long long a = gemm_cost(pg), b = sketch_cost(total - pg);
+    const long long c = (a > b ? a : b) + 1500;      // fork and join
+    if (c < best_cost) { best_cost = c; best.gemm_pairs = pg; best.sketch_clusters = total - pg; }
+  }
+  return best;
+}
+
+// Runs `on_side` on a side stream that starts after everything queued on `stream` so far and that `stream` waits for
+// afterwards; `on_main` is queued on `stream` in between.
+template <class FSide, class FMain>
+rmm_status fork_join(cudaStream_t stream, FSide&& on_side, FMain&& on_main) {
+  DeviceState& ds = device_state();
+  const unsigned lane = ds.next_lane.fetch_add(1) % DeviceState::kLanes;
+  std::lock_guard<std::mutex> lock(ds.lane_mutex[lane]);
+  cudaStream_t side = ds.lane_stream[lane];
+  if (cudaEventRecord(ds.lane_fork[lane], stream) != cudaSuccess) return RMM_ERR_CUDA;
+  if (cudaStreamWaitEvent(side, ds.lane_fork[lane], 0) != cudaSuccess) return RMM_ERR_CUDA;
+  rmm_status st = on_side(side);
+  // the join is queued even after an error, so that the side stream never runs ahead of the caller's stream
+  const bool rec = cudaEventRecord(ds.lane_join[lane], side) == cudaSuccess;
+  const rmm_status st2 = on_main(stream);
+  const bool wait = rec && cudaStreamWaitEvent(stream, ds.lane_join[lane], 0) == cudaSuccess;
+  if (st != RMM_OK) return st;
+  if (st2 != RMM_OK) return st2;
+  return wait ? RMM_OK : RMM_ERR_CUDA;
+}
+
+std::atomic<int> g_pass_mode{0};
 
 // ------------------------------------------------------------------ allocation-free bias gradient
 // Scratch for rmm_bias_grad_static: partial column sums, [slice][column].  The name below
@@ -437,15 +767,46 @@ rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, i
   const float c = sketch_scale(B_proj, dist);
 
   if (dt == RMM_DTYPE_BF16) {
+    float* scratch = reinterpret_cast<float*>(ws + w.scratch_off);
+    const size_t scratch_bytes = w.total - w.scratch_off;
     // the first kernel of the call resets the status word (no separate memset on the stream)
-    if (Y) {
-      ScopedTiming t(RMM_STEP_Y, stream);
-      st = launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, status, stream, nullptr, true);
-      if (st != RMM_OK) return st;
+    if (dist == RMM_DIST_SORS_HADAMARD && sors_fast_supported(B_proj, D_in, N, scratch_bytes)) {
+      // the subsampled-Hadamard sketch by its fast transform; the dense product on its own
+      if (Y) {
+        ScopedTiming t(RMM_STEP_Y, stream);
+        st = launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, status, stream, nullptr, true);
+        if (st != RMM_OK) return st;
+      }
+      ScopedTiming t(RMM_STEP_SKETCH, stream);
+      return launch_sors_fast(X, X_proj, nullptr, B_proj, D_in, N, c, pk, scratch, scratch_bytes, status, stream, Y == nullptr);
     }
-    ScopedTiming t(RMM_STEP_SKETCH, stream);
-    return launch_sketch(X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, reinterpret_cast<float*>(ws + w.scratch_off),
-                         status, stream, Y == nullptr, w.total - w.scratch_off);
+    if (g_pass_mode.load(std::memory_order_relaxed) == 1) {
+      // Y = X W^T + 1 b^T and X_proj = S^T X in one launch
+      ScopedTiming t(RMM_STEP_FWD, stream);
+      PassArgs a;
+      if (Y) { a.a = X; a.b = W; a.bias = b; a.c = Y; a.M = N; a.N = D_out; a.K = D_in; a.bmode = tc::B_K; }
+      a.data = X; a.out = X_proj; a.k = B_proj; a.cols = D_in; a.tokens = N; a.scale = c; a.dist = (int)dist;
+      return launch_pass(a, pk, scratch, reinterpret_cast<unsigned long long*>(ws + w.ticket_off), status, stream, true);
+    }
+    if (!Y) {
+      ScopedTiming t(RMM_STEP_SKETCH, stream);
+      return launch_sketch(X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, scratch, status, stream, true);
+    }
+    // Y = X W^T + 1 b^T and X_proj = S^T X: two kernels that share the device and the X stream
+    const PassSplit split = plan_pass_split(N, D_out, D_in, B_proj, D_in, N);
+    ScopedTiming t(RMM_STEP_FWD, stream);
+    auto gemm = [&](cudaStream_t s_, int pairs) {
+      return launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, status, s_, nullptr, true, pairs);
+    };
+    auto sketch = [&](cudaStream_t s_, int clusters) {
+      return launch_sketch(X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, scratch, status, s_, false, clusters);
+    };
+    if (split.gemm_pairs == 0) {
+      st = gemm(stream, 0);
+      return st != RMM_OK ? st : sketch(stream, 0);
+    }
+    return fork_join(stream, [&](cudaStream_t side) { return sketch(side, split.sketch_clusters); },
+                     [&](cudaStream_t main_) { return gemm(main_, split.gemm_pairs); });
   }
   if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return RMM_ERR_CUDA;
   if (Y) {
@@ -476,17 +837,48 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
   const float c = sketch_scale(B_proj, dist);
 
   if (dt == RMM_DTYPE_BF16) {
+    float* scratch = reinterpret_cast<float*>(ws + w.scratch_off);
+    const size_t scratch_bytes = w.total - w.scratch_off;
     // the first kernel of the call resets the status word (no separate memset on the stream)
-    if (dX) {
-      ScopedTiming t(RMM_STEP_DX, stream);
-      st = launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, status, stream, nullptr, true);
-      if (st != RMM_OK) return st;
-    }
-    {
-      // db = dY^T 1 comes out of the same contraction as the extra row of ones of S^T
+    if (dist == RMM_DIST_SORS_HADAMARD && sors_fast_supported(B_proj, D_out, N, scratch_bytes)) {
+      if (dX) {
+        ScopedTiming t(RMM_STEP_DX, stream);
+        st = launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, status, stream, nullptr, true);
+        if (st != RMM_OK) return st;
+      }
       ScopedTiming t(RMM_STEP_SDY, stream);
-      st = launch_sketch(dY, G, db, B_proj, D_out, N, c, dist, pk, reinterpret_cast<float*>(ws + w.scratch_off), status,
-                         stream, dX == nullptr, w.total - w.scratch_off);
+      st = launch_sors_fast(dY, G, db, B_proj, D_out, N, c, pk, scratch, scratch_bytes, status, stream, dX == nullptr);
+      if (st != RMM_OK) return st;
+    } else if (g_pass_mode.load(std::memory_order_relaxed) == 1) {
+      // dX = dY W, G = S^T dY and db = dY^T 1 (the row of ones of S^T) in one launch
+      ScopedTiming t(RMM_STEP_BWD, stream);
+      PassArgs a;
+      if (dX) { a.a = dY; a.b = W; a.c = dX; a.M = N; a.N = D_in; a.K = D_out; a.bmode = tc::B_MN; }
+      a.data = dY; a.out = G; a.ones_out = db; a.k = B_proj; a.cols = D_out; a.tokens = N; a.scale = c; a.dist = (int)dist;
+      st = launch_pass(a, pk, scratch, reinterpret_cast<unsigned long long*>(ws + w.ticket_off), status, stream, true);
+      if (st != RMM_OK) return st;
+    } else if (!dX) {
+      ScopedTiming t(RMM_STEP_SDY, stream);
+      st = launch_sketch(dY, G, db, B_proj, D_out, N, c, dist, pk, scratch, status, stream, true);
+      if (st != RMM_OK) return st;
+    } else {
+      // dX = dY W and G = S^T dY (with db = dY^T 1 as the row of ones of S^T): two kernels that share the device and
+      // the dY stream
+      const PassSplit split = plan_pass_split(N, D_in, D_out, B_proj + 1, D_out, N);
+      ScopedTiming t(RMM_STEP_BWD, stream);
+      auto gemm = [&](cudaStream_t s_, int pairs) {
+        return launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, status, s_, nullptr, true, pairs);
+      };
+      auto sketch = [&](cudaStream_t s_, int clusters) {
+        return launch_sketch(dY, G, db, B_proj, D_out, N, c, dist, pk, scratch, status, s_, false, clusters);
+      };
+      if (split.gemm_pairs == 0) {
+        st = gemm(stream, 0);
+        if (st == RMM_OK) st = sketch(stream, 0);
+      } else {
+        st = fork_join(stream, [&](cudaStream_t side) { return sketch(side, split.sketch_clusters); },
+                       [&](cudaStream_t main_) { return gemm(main_, split.gemm_pairs); });
+      }
       if (st != RMM_OK) return st;
     }
     ScopedTiming t(RMM_STEP_DW, stream);
@@ -571,6 +963,19 @@ int64_t rmm_debug_sketch_schedule(int64_t rows, int64_t cols, int64_t tokens, in
     for (int tile = 0; tile < sc.tiles(); ++tile)
       tc::sketch_for_each_slot_of_tile(sc, tile, [&](long long slot) { put(tile, slot, 0, 0, 0); });
   }
+  return n;
+}
+
+int64_t rmm_debug_pass_schedule(int64_t gemm_m, int64_t gemm_n, int64_t gemm_k, int64_t rows, int64_t cols, int64_t tokens,
+                                int max_pairs, int64_t* out, int64_t cap) {
+  if (max_pairs < 1 || gemm_m < 0 || rows < 0) return -1;
+  const bool with_gemm = gemm_m > 0, with_sketch = rows > 0;
+  if (with_gemm && (gemm_n < 1 || gemm_k < 1)) return -1;
+  if (with_sketch && (cols < 1 || tokens < 1)) return -1;
+  const tc::PassSchedule s = make_pass_schedule(with_gemm, gemm_m, gemm_n, gemm_k, with_sketch, rows, cols, tokens, max_pairs);
+  const int64_t head[10] = {s.num_pairs, s.gemm_tiles, s.tiles_n, s.num_kb, s.tiles_m, s.groups, s.nat, s.ksteps, s.nb, s.blen};
+  const int64_t n = 10 + s.num_pairs + 1;
+  for (int64_t i = 0; i < n && i < cap && out; ++i) out[i] = i < 10 ? head[i] : s.gemm_begin[i - 10];
   return n;
 }
 
@@ -679,6 +1084,22 @@ rmm_status rmm_bias_grad_static(const void* dY, int64_t N, int64_t D_out, rmm_dt
   }
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
 }
+
+#ifdef RMM_PASS_TRACE
+// Trace build only: copies the cycle counters of the last pass launch ([148][32] int64) to host memory.
+int rmm_debug_pass_trace(long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, tc::g_pass_trace, sizeof(long long) * 2 * tc::PS_MAX_PAIRS * tc::PS_TRACE_SLOTS) ==
+                 cudaSuccess ? 0 : 1;
+}
+#endif
+
+rmm_status rmm_set_pass_mode(int mode) {
+  if (mode != 0 && mode != 1) return RMM_ERR_INVALID_ARG;
+  g_pass_mode.store(mode, std::memory_order_relaxed);
+  return RMM_OK;
+}
+
+int64_t rmm_layer_launch_count(void) { return (int64_t)g_layer_launches.load(std::memory_order_relaxed); }
 
 rmm_status rmm_profile_enable(int capacity) {
   Profiler& p = profiler();

@@ -107,6 +107,13 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// The same with the default semantics of mbarrier.arrive (release at CTA scope): for a producer that has made its
+// shared-memory writes visible to the async proxy (fence_proxy_async_smem) and whose data is read by the tensor
+// cores, not by the threads that wait on the barrier.  A cluster-scope release makes the arriving thread wait
+// until all its earlier writes are visible cluster-wide, which costs thousands of cycles per arrival.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 // Asynchronous copy of `bytes` (a multiple of 16, both addresses 16-byte aligned) from this CTA's
 // shared memory into the shared memory of a CTA of the cluster (address from mapa_shared). The
 // bytes are counted on an mbarrier of the destination CTA, so the consumer's wait on that barrier
@@ -193,6 +200,22 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc,
 // arrive on a barrier (of any CTA of the cluster) once all pair MMAs issued so far have completed
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr)
+               : "memory");
+}
+
+// The same arrival on the barriers at this shared-memory offset in every CTA of the pair named by `cta_mask`
+// (bit r = CTA of rank r), with one instruction.
+__device__ __forceinline__ void umma_commit_pair_multicast(uint32_t bar_local_addr, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar_local_addr), "h"(cta_mask)
+               : "memory");
+}
+// Asynchronous 4-byte store into the shared memory of a CTA of the cluster whose 4 bytes are counted on an mbarrier of
+// that CTA (both addresses from mapa_shared).  Does not block the issuing thread: used as a signal across the pair
+// where an mbarrier.arrive on a shared::cluster address stalls the arriving warp for thousands of cycles.
+__device__ __forceinline__ void st_async_u32(uint32_t dst_cluster_addr, uint32_t value, uint32_t cluster_mbar) {
+  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+               ::"r"(dst_cluster_addr), "r"(value), "r"(cluster_mbar)
                : "memory");
 }
 

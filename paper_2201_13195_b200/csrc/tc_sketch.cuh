@@ -92,6 +92,7 @@ struct SketchSchedule {
   int w_last;              // width of the last block (0 if none)
   int upl;                 // units per CTA in the last block's line
   long long lcm_last;      // lcm(upl, w_last)
+  long long est_steps;     // host only: estimated time of the busiest cluster, in 64-token steps (drains included)
 
   __host__ __device__ int tiles() const { return tiles_m * tiles_n; }
   __host__ __device__ long long num_slots() const { return (long long)tiles() + num_ctas; }
@@ -212,6 +213,7 @@ inline SketchSchedule make_sketch_schedule(long long rows, long long cols, long 
   s.tiles_rem = tiles % max_ctas;
   s.num_ctas = max_ctas;
   s.upc = 0; s.full_blocks = 0; s.w_last = 0; s.upl = 1; s.lcm_last = 1;
+  s.est_steps = (long long)s.rounds * (s.ksteps + 14);
   if (s.tiles_rem > 0) {
     // Every segment ends with a drain of the accumulator that the next segment has to wait for:
     // about kSegCost steps' worth.  CTAs of the last block's line work on several tiles, so they
@@ -257,6 +259,7 @@ inline SketchSchedule make_sketch_schedule(long long rows, long long cols, long 
         }
       }
     }
+    s.est_steps += best_cost;
     if (s.w_last > 0) s.lcm_last = (long long)s.upl / gcd_ll(s.upl, s.w_last) * s.w_last;
     const long long last_ctas = s.w_last > 0 ? ((long long)s.tiles_rem * s.w_last + s.upl - 1) / s.upl : 0;
     const long long used = (long long)s.full_blocks * s.tiles_rem + last_ctas;

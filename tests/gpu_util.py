@@ -79,9 +79,16 @@ def oracle_layer(w: R.Workload, inputs, gpu_xproj=None):
 #     end to end, where the oracle's X_proj is not rounded either, by twice that (first order).
 #   fp32 mode: |got - r| <= 2^-20 |r| + sqrt(K) 2^-19 rms (fp32 FMA chain of length K: rounding errors of size
 #     2^-24 times the partial sums, adding up like a random walk; sixteen times that as the allowance).
+#   Subsampled-Hadamard sketch in bf16 mode (applied by the two-level Walsh-Hadamard transform): the first
+#     level's result T is stored in bf16, so every element of X_proj and of G carries one more rounding whose
+#     sum over the L/128 blocks has standard deviation 2^-9/sqrt(3) sqrt(L/N) rms <= 1.6e-3 rms (L = Hadamard
+#     order < 2N), whatever the element's size: 2^-6 rms (ten standard deviations) is added for X_proj and dW.
 # A wrong element (a mis-clipped store box, a stale 16-byte chunk, a missing partial tile) is off by the order
 # of rms and fails this gate by an order of magnitude or more, while it passes the Frobenius gate.
-def elementwise_excess(got, ref, dtype, K, operand_term=None):
+SORS_FAST_PATH_EXTRA = 2.0 ** -6
+
+
+def elementwise_excess(got, ref, dtype, K, operand_term=None, extra_rms=0.0):
     """max over elements of |got - ref| / bound; <= 1 passes.  Returns (excess, index of the worst element)."""
     got, ref = np.asarray(got, np.float64), np.asarray(ref, np.float64)
     assert got.shape == ref.shape
@@ -92,7 +99,7 @@ def elementwise_excess(got, ref, dtype, K, operand_term=None):
         rel, a = 2.0 ** -8, 2.0 ** -10 + K * 2.0 ** -23
     else:
         rel, a = 2.0 ** -20, np.sqrt(K) * 2.0 ** -19
-    bound = rel * np.abs(ref) + a * rms + 1e-300
+    bound = rel * np.abs(ref) + (a + extra_rms) * rms + 1e-300
     if operand_term is not None:
         bound = bound + operand_term
     ratio = np.abs(got - ref) / bound
@@ -112,7 +119,7 @@ def contraction_lengths(N, d_in, d_out, k):
     return {"Y": d_in, "X_proj": N, "dX": d_out, "dW": k, "db": N}
 
 
-def assert_parity(got, ref, dtype, names=("Y", "X_proj", "dX", "dW", "db"), K=None, end_to_end=False):
+def assert_parity(got, ref, dtype, names=("Y", "X_proj", "dX", "dW", "db"), K=None, end_to_end=False, dist=None):
     """Relative Frobenius error per tensor within TOL and, when the contraction lengths K are given, every
     element within the element-wise bound above (ref must then hold the oracle's G and X_proj as well)."""
     errs = {n: O.rel_frobenius(got[n], ref[n]) for n in names}
@@ -121,7 +128,8 @@ def assert_parity(got, ref, dtype, names=("Y", "X_proj", "dX", "dW", "db"), K=No
     if K is not None:
         for n in names:
             term = dw_operand_term(ref["G"], ref["X_proj_used"], dtype, end_to_end) if n == "dW" else None
-            ex, where = elementwise_excess(got[n], ref[n], dtype, K[n], term)
+            extra = SORS_FAST_PATH_EXTRA if (dist == R.DIST_SORS and dtype == R.DTYPE_BF16 and n in ("X_proj", "dW")) else 0.0
+            ex, where = elementwise_excess(got[n], ref[n], dtype, K[n], term, extra)
             assert ex <= 1.0, f"{n}{list(where)}: |got - ref| is {ex:.2f} x its element-wise bound " \
                               f"(got {np.asarray(got[n])[where]}, ref {np.asarray(ref[n])[where]})"
     return errs

@@ -177,3 +177,37 @@ def test_variance_probe_argument_errors(lib):
     import torch
     if not torch.cuda.is_available():
         assert probe(p, p, 16, 8, 8, 4, 0, 0, p, None, p, 1 << 30, None) == CUDA        # no device: an error, no fallback
+
+
+@pytest.mark.parametrize("N,d_in,d_out,k,pairs", [
+    (16384, 1024, 4096, 1638, 74), (16384, 4096, 1024, 1638, 74), (4096, 768, 3072, 819, 74), (4096, 768, 3072, 3686, 74),
+    (4096, 3072, 768, 819, 74), (4096, 768, 2304, 819, 74), (4096, 768, 768, 819, 74), (37, 24, 40, 5, 74),
+    (1, 8, 8, 1, 74), (300, 264, 520, 130, 74), (9700, 512, 64, 16, 74), (19200, 1024, 64, 16, 74),
+    (2900, 4096, 64, 2816, 74), (16384, 1024, 4096, 1638, 5), (4096, 768, 3072, 819, 1), (100000, 64, 64, 16, 74),
+])
+def test_pass_schedule_covers_all_work_and_fits_the_workspace(N, d_in, d_out, k, pairs):
+    """Host logic of the one-launch passes: every dense tile belongs to exactly one pair, the token blocks of a
+    sketch tile cover its steps exactly once, no pair index is out of range, and the partial tiles fit the
+    scratch part of the workspace that rmm_workspace_bytes asks for."""
+    import paper_2201_13195_b200 as P
+    ws = P.rmm_workspace_bytes(N, d_in, d_out, k, P.RMM_DTYPE_BF16)
+    for gemm, sketch in (((N, d_out, d_in), (k, d_in, N)), ((N, d_in, d_out), (k + 1, d_out, N)),
+                         (None, (k, d_in, N)), ((N, d_out, d_in), None)):
+        s = P.rmm_debug_pass_schedule(gemm, sketch, pairs)
+        assert 1 <= s["num_pairs"] <= pairs
+        gb = s["gemm_begin"]
+        assert gb[0] == 0 and gb[-1] == s["gemm_tiles"] and all(a <= b for a, b in zip(gb, gb[1:]))
+        if gemm:
+            assert s["gemm_tiles"] == -(-gemm[0] // 256) * -(-gemm[1] // 256) and s["num_kb"] == -(-gemm[2] // 64)
+        else:
+            assert s["gemm_tiles"] == 0
+        if sketch:
+            rows, cols, tokens = sketch
+            assert s["tiles_m"] == -(-rows // 128) and s["ksteps"] == -(-tokens // 64)
+            assert 1 <= s["nat"] <= 4 and s["groups"] * s["nat"] * 256 >= cols > (s["groups"] - 1) * s["nat"] * 256
+            assert (s["nb"] - 1) * s["blen"] < s["ksteps"] <= s["nb"] * s["blen"]      # blocks: non-empty, cover all steps
+            units = s["tiles_m"] * s["groups"] * s["nb"]
+            assert units * 128 * s["nat"] * 256 * 4 <= ws                             # partial tiles fit the workspace
+            assert s["num_pairs"] == min(pairs, units + s["gemm_tiles"])
+        else:
+            assert s["tiles_m"] == 0
