@@ -86,8 +86,10 @@ Workspace workspace_layout(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rm
   size_t scratch = (size_t)w.db_slices * (size_t)D_out * sizeof(float);
   if (dt == RMM_DTYPE_BF16) {
     // an upper bound over every grid the launch may use: one partial tile per (tile, CTA) pair at most
-    const long long tf = ((k + tc::SK_BM - 1) / tc::SK_BM) * ((D_in + tc::SK_BN - 1) / tc::SK_BN);
-    const long long tb = ((k + 1 + tc::SK_BM - 1) / tc::SK_BM) * ((D_out + tc::SK_BN - 1) / tc::SK_BN);
+    // (512-column blocks are counted in pairs: a cluster of two CTAs has a slot for each of its CTAs)
+    auto blocks2 = [](int64_t d) { const int64_t b = (d + tc::SK_BN - 1) / tc::SK_BN; return b >= 2 ? (b + 1) / 2 * 2 : b; };
+    const long long tf = ((k + tc::SK_BM - 1) / tc::SK_BM) * blocks2(D_in);
+    const long long tb = ((k + 1 + tc::SK_BM - 1) / tc::SK_BM) * blocks2(D_out);
     scratch = (size_t)((tf > tb ? tf : tb) + tc::SK_MAX_CTAS) * tc::SK_TILE_ELEMS * sizeof(float);
     if (scratch_pass > scratch) scratch = scratch_pass;
   }
@@ -402,7 +404,7 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
                          bool clear_status = false, int clusters_limit = 0) {
   CUtensorMap tmB;
   const bool slab_map = cols % 64 == 0;
-  if (!(slab_map ? make_tmap_slabs(&tmB, b, tokens, cols, tc::SK_BK, tc::SK_BN / 64)
+  if (!(slab_map ? make_tmap_slabs(&tmB, b, tokens, cols, tc::SK_BK, tc::SK_BNH / 64)
                  : make_tmap(&tmB, b, tokens, cols, tc::SK_BK)))
     return RMM_ERR_CUDA;
   tc::SketchParams p;
@@ -1088,7 +1090,7 @@ rmm_status rmm_bias_grad_static(const void* dY, int64_t N, int64_t D_out, rmm_dt
 #ifdef RMM_PASS_TRACE
 // Trace build only: copies the cycle counters of the last pass launch ([148][32] int64) to host memory.
 int rmm_debug_pass_trace(long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, tc::g_pass_trace, sizeof(long long) * 2 * tc::PS_MAX_PAIRS * tc::PS_TRACE_SLOTS) ==
+  return cudaMemcpyFromSymbol(host_out, tc::g_pass_trace, sizeof(long long) * 148 * tc::PS_TRACE_SLOTS) ==
                  cudaSuccess ? 0 : 1;
 }
 #endif

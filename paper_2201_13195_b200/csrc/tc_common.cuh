@@ -305,6 +305,22 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t v[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Optional cycle accounting (build with -DRMM_PASS_TRACE): per CTA, how long each role spent in its loops
+// and in each kind of wait.  Read back with rmm_debug_pass_trace.  Not compiled into the product library.
+#ifdef RMM_PASS_TRACE
+constexpr int PS_TRACE_SLOTS = 32;
+__device__ long long g_pass_trace[148][PS_TRACE_SLOTS];
+#define PS_TRACE_DECL(name) long long name = 0
+#define PS_TRACE_T0(name) const long long name = clock64()
+#define PS_TRACE_ADD(acc, t0) acc += clock64() - (t0)
+#define PS_TRACE_PUT(slot, value) g_pass_trace[blockIdx.x][slot] = (value)
+#else
+#define PS_TRACE_DECL(name)
+#define PS_TRACE_T0(name)
+#define PS_TRACE_ADD(acc, t0)
+#define PS_TRACE_PUT(slot, value)
+#endif
+
 // ---------------------------------------------------------------- descriptors
 // Shared-memory matrix descriptor, 128-byte swizzle.  Bits: [0,14) start address >> 4,
 // [16,30) leading byte offset >> 4, [32,46) stride byte offset >> 4, [46,48) version = 1,

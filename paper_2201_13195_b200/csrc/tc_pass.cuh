@@ -184,23 +184,8 @@ __device__ __forceinline__ bool ticket_wait(const unsigned long long* t, unsigne
   return false;
 }
 
-// Optional cycle accounting (build with -DRMM_PASS_TRACE): per CTA, how long each role spent in its loops
-// and in each kind of wait.  Read back with rmm_debug_pass_trace.  Not compiled into the product library.
 #ifndef PS_EXP_GUARD
 #define PS_EXP_GUARD
-#endif
-#ifdef RMM_PASS_TRACE
-constexpr int PS_TRACE_SLOTS = 32;
-__device__ long long g_pass_trace[2 * PS_MAX_PAIRS][PS_TRACE_SLOTS];
-#define PS_TRACE_DECL(name) long long name = 0
-#define PS_TRACE_T0(name) const long long name = clock64()
-#define PS_TRACE_ADD(acc, t0) acc += clock64() - (t0)
-#define PS_TRACE_PUT(slot, value) g_pass_trace[blockIdx.x][slot] = (value)
-#else
-#define PS_TRACE_DECL(name)
-#define PS_TRACE_T0(name)
-#define PS_TRACE_ADD(acc, t0)
-#define PS_TRACE_PUT(slot, value)
 #endif
 // trace slots: 0 kernel cycles; producer: 1 wait empty, 2 loop; MMA: 3 wait S^T, 4 wait data, 5 wait accumulator,
 // 6 sketch loop, 7 dense loop; generator warp 6: 8 arithmetic, 9 wait free stage, 10 loop; warp 2: 11 wait sketch

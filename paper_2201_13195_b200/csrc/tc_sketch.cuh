@@ -48,11 +48,13 @@
 namespace rmm {
 namespace tc {
 
-constexpr int SK_BM = 128, SK_BN = 512, SK_AK = 64, SK_BK = 32;
+constexpr int SK_BM = 128, SK_BN = 512, SK_AK = 64;
+constexpr int SK_BK = 64;                            // tokens of a B stage
+constexpr int SK_BNH = 256;                          // columns of a B stage: one half of the tile, one MMA warp's
 constexpr int SK_A_STAGES = 3, SK_B_STAGES = 5;
 constexpr int SK_A_BYTES = SK_BM * SK_AK * 2;        // 16 KiB
-constexpr int SK_B_BYTES = SK_BN * SK_BK * 2;        // 32 KiB
-constexpr int SK_B_SLAB = 64 * SK_BK * 2;            // [32 tokens][64 columns] = 4 KiB
+constexpr int SK_B_BYTES = SK_BNH * SK_BK * 2;       // 32 KiB
+constexpr int SK_B_SLAB = 64 * SK_BK * 2;            // [64 tokens][64 columns] = 8 KiB
 constexpr int SK_STAGGER = 2;                        // steps by which neighbouring tile rows are offset
 constexpr int SK_GEN_GROUPS = SK_A_STAGES;  // one generator warp group per ring stage: group g fills stage g.
 // (A stage must have one producer group: barrier waits only see the parity of a phase, and two
@@ -195,11 +197,12 @@ __host__ __device__ inline void sketch_for_each_slot_of_tile(const SketchSchedul
 
 inline long long gcd_ll(long long a, long long b) { while (b) { long long t = a % b; a = b; b = t; } return a; }
 
-// Cluster size for a result with `cols` columns: the largest of 4, 2, 1 that divides the number
-// of 512-column blocks.
+// Cluster size for a result with `cols` columns: two CTAs (neighbouring 512-column blocks) share every
+// generated S^T stage whenever there are at least two blocks.  With an odd number of blocks the last cluster's
+// second CTA has no columns of its own: it still generates and sends its half of S^T, and skips the rest.
 inline int sketch_cluster_size(long long cols) {
   const long long blocks = (cols + SK_BN - 1) / SK_BN;
-  return blocks % 2 == 0 ? 2 : 1;
+  return blocks >= 2 ? 2 : 1;
 }
 
 inline SketchSchedule make_sketch_schedule(long long rows, long long cols, long long tokens, int cluster, int max_ctas) {
@@ -351,6 +354,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
   static_assert(SK_GEN_WARPS % SK_GEN_GROUPS == 0 && TASKS % GROUP_THREADS == 0, "generator groups");
 
   MBAR_PEEK_DECLARE();
+  PS_TRACE_T0(trace_kernel0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = (C == 1) ? 0u : cluster_ctarank();
   const SketchSchedule& sc = p.sched;
@@ -365,7 +369,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     }
     for (int s = 0; s < SK_B_STAGES; ++s) {
       mbar_init(fullb_bar(s), 1);
-      mbar_init(emptyb_bar(s), SK_MMA_WARPS);
+      mbar_init(emptyb_bar(s), 1);              // a B stage belongs to one MMA warp
     }
     mbar_init(accfull_bar, SK_MMA_WARPS);
     mbar_init(accempty_bar, SK_GEN_WARPS);
@@ -391,113 +395,156 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       int seg_it = 0;
       long long cursor = 0;
       SketchSegment sg;
+      PS_TRACE_DECL(tr_pw);
+      PS_TRACE_T0(tr_pl);
       while (ok && sketch_next_segment(sc, cl, seg_it, cursor, sg)) {
         const int n0 = ((sg.tile % sc.tiles_n) * C + (int)rank) * SK_BN;
         for (int i = 0; i < sg.ks1 - sg.ks0 && ok; ++i) {
           const int ks = sketch_step(sg.ks0, sg.ks1, sg.tile / sc.tiles_n, i);
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
+          for (int nh = 0; nh < 2; ++nh) {       // one stage per column half: 64 tokens x 256 columns
+            if (n0 + nh * SK_BNH >= p.cols) continue;      // no such columns: the MMA warp of this half skips it too
+            PS_TRACE_T0(tw);
             if (!mbar_wait(emptyb_bar(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            PS_TRACE_ADD(tr_pw, tw);
             const uint32_t b_smem = smem_u32(b_ring) + s * SK_B_BYTES;
             mbar_arrive_expect_tx(fullb_bar(s), SK_B_BYTES);
-            const int tok0 = ks * SK_AK + half * SK_BK;
+            const int tok0 = ks * SK_AK;
+            const int c0 = n0 + nh * SK_BNH;
             if (p.slab_map) {
-              // one instruction for all eight [32 tokens][64 columns] slabs of the stage
-              tma_load_3d(b_smem, &tmB, fullb_bar(s), 0, tok0, n0 >> 6);
+              // one instruction for all four [64 tokens][64 columns] slabs of the stage
+              tma_load_3d(b_smem, &tmB, fullb_bar(s), 0, tok0, c0 >> 6);
             } else {
 #pragma unroll
-              for (int sl = 0; sl < SK_BN / 64; ++sl)
-                tma_load_2d(b_smem + sl * SK_B_SLAB, &tmB, fullb_bar(s), n0 + 64 * sl, tok0);
+              for (int sl = 0; sl < SK_BNH / 64; ++sl)
+                tma_load_2d(b_smem + sl * SK_B_SLAB, &tmB, fullb_bar(s), c0 + 64 * sl, tok0);
             }
             if (++s == SK_B_STAGES) { s = 0; ph ^= 1u; }
           }
         }
       }
+      PS_TRACE_PUT(1, tr_pw);
+      PS_TRACE_PUT(2, clock64() - tr_pl);
     }
     __syncwarp();
   } else if (warp <= SK_MMA_WARPS) {
     // ------------------------------------------------------------ MMA issuers
-    // Two warps, one per 256-column half of the accumulator: the issue loop is a serial chain of
-    // barrier waits, descriptor arithmetic, MMAs and commits, and one warp alone does not get
-    // through a K-step in the time the tensor pipe needs for it.  Both wait on the same full
-    // barriers; a stage is free once both have committed.
+    // Two warps, one per 256-column half of the accumulator.  The tensor pipe needs 128 cycles per MMA
+    // (M 128 x N 256 x K 16); the issuing thread shares its scheduler with three generator warps, so its
+    // loop is kept short: one barrier round (test, fence, election, commits) per four MMAs, each warp with
+    // B stages of its own (64 tokens x its 256 columns), descriptors that differ only in the low word.
+    // Both warps read the same S^T stages; an S^T stage is free once both (in every CTA) have committed.
     const int nh = warp - 1;
     // The whole warp runs the loop, so that descriptors and addresses stay warp-uniform (the
     // tcgen05 operands live in uniform registers); one elected lane issues.
     {
-      constexpr uint32_t idesc = instr_desc_bf16(SK_BM, 256, false, true);
-      // Descriptors are built once, stage and K-step offsets are added to the start-address
-      // field (16-byte units).
+      constexpr uint32_t idesc = instr_desc_bf16(SK_BM, SK_BNH, false, true);
+      // Descriptors are built once; stage and K-step offsets are added to the start-address field (16-byte
+      // units, 14 bits: no carry into the high word).
       const uint64_t adesc0 = smem_desc_sw128(smem_u32(a_ring), 16, 1024);
       const uint64_t bdesc0 = smem_desc_sw128(smem_u32(b_ring), SK_B_SLAB, 1024);
+      const uint32_t a_lo0 = (uint32_t)adesc0, a_hi = (uint32_t)(adesc0 >> 32);
+      const uint32_t b_lo0 = (uint32_t)bdesc0, b_hi = (uint32_t)(bdesc0 >> 32);
+      auto desc64 = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | (uint64_t)lo; };
       uint32_t peer_emptya0[C];                  // emptyA[0] of every CTA of the cluster
 #pragma unroll
       for (int r = 0; r < C; ++r) peer_emptya0[r] = (C == 1) ? emptya_bar(0) : mapa_shared(emptya_bar(0), r);
-      int sa = 0, sb = 0;
-      uint32_t pha = 0, phb = 0;
+      // B ring: the producer fills one stage per step and column half that exists (a half that starts beyond
+      // the last column is skipped); qs / qph = ring position and phase of the step's first stage.
+      int sa = 0, qs = 0;
+      uint32_t pha = 0, qph = 0;
       int seg = 0;
       bool ok = true;
+      bool bpeek = false;                        // the B barrier of the coming step has been tested
       int seg_it = 0;
       long long cursor = 0;
       SketchSegment sg;
       // Each full barrier is tested one stage ahead (slot 0: S^T ring, slot 1: B ring).
       if (C == 1) { MBAR_PEEK(0, fulla_bar(0), 0u); } else { MBAR_PEEK_CLUSTER(0, fulla_bar(0), 0u); }
-      MBAR_PEEK(1, fullb_bar(0), 0u);
+      PS_TRACE_DECL(tr_ws);
+      PS_TRACE_DECL(tr_wd);
+      PS_TRACE_DECL(tr_wa);
+      PS_TRACE_DECL(tr_m_is);
+      PS_TRACE_DECL(tr_m_co);
+      PS_TRACE_T0(tr_sk0);
       for (; ok && sketch_next_segment(sc, cl, seg_it, cursor, sg); ++seg) {
+        const long long n0 = (long long)((sg.tile % sc.tiles_n) * C + (int)rank) * SK_BN;
+        const int live0 = n0 < p.cols ? 1 : 0, live1 = n0 + SK_BNH < p.cols ? 1 : 0;
+        const bool mine = nh == 0 ? live0 != 0 : live1 != 0;      // this warp's half has columns
+        const int myoff = (nh == 1 && live0) ? 1 : 0;
         if (seg > 0) {   // the previous segment's accumulator must have been drained
+          PS_TRACE_T0(tw);
           ok = (mbar_wait_warp(accempty_bar, (uint32_t)(seg - 1) & 1u, abort_flag, p.status));
+          PS_TRACE_ADD(tr_wa, tw);
           if (!ok) break;
           tc_fence_after();
         }
         uint32_t acc = 0;
+        bpeek = false;
         for (int ks = sg.ks0; ks < sg.ks1 && ok; ++ks) {
           uint32_t ready;
           MBAR_PEEK_RESULT(0, ready);
           if (!__all_sync(0xffffffffu, ready != 0)) {
+            PS_TRACE_T0(tw);
             ok = (C == 1) ? mbar_wait_warp(fulla_bar(sa), pha, abort_flag, p.status)
                           : mbar_wait_cluster_warp(fulla_bar(sa), pha, abort_flag, p.status);
+            PS_TRACE_ADD(tr_ws, tw);
             if (!ok) break;
           }
-          const uint64_t ad = adesc0 + (uint64_t)(sa * (SK_A_BYTES >> 4));
           const int sa_next = (sa + 1 == SK_A_STAGES) ? 0 : sa + 1;
           const uint32_t pha_next = (sa_next == 0) ? (pha ^ 1u) : pha;
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            MBAR_PEEK_RESULT(1, ready);
+          int sb = qs + myoff;
+          uint32_t phb = qph;
+          if (sb >= SK_B_STAGES) { sb -= SK_B_STAGES; phb ^= 1u; }
+          int qn = qs + live0 + live1;
+          uint32_t qphn = qph;
+          if (qn >= SK_B_STAGES) { qn -= SK_B_STAGES; qphn ^= 1u; }
+          bool issuer = false;
+          if (mine) {
+            ready = 0;
+            if (bpeek) MBAR_PEEK_RESULT(1, ready);
             if (!__all_sync(0xffffffffu, ready != 0)) {
+              PS_TRACE_T0(tw);
               ok = (mbar_wait_warp(fullb_bar(sb), phb, abort_flag, p.status));
+              PS_TRACE_ADD(tr_wd, tw);
               if (!ok) break;
             }
             tc_fence_after();
-            const uint64_t bd = bdesc0 + (uint64_t)(sb * (SK_B_BYTES >> 4));
-            const int sb_next = (sb + 1 == SK_B_STAGES) ? 0 : sb + 1;
-            const uint32_t phb_next = (sb_next == 0) ? (phb ^ 1u) : phb;
-            const bool issuer = elect_one();
+            const uint32_t a_lo = a_lo0 + (uint32_t)(sa * (SK_A_BYTES >> 4));
+            const uint32_t b_lo = b_lo0 + (uint32_t)(sb * (SK_B_BYTES >> 4));
+            PS_TRACE_T0(tis);
+            issuer = elect_one();
             if (issuer) {
 #pragma unroll
-              for (int j = 0; j < SK_BK / 16; ++j) {
-                umma_bf16(tmem_base + nh * 256, ad + (half * (SK_BK / 16) + j) * 2,
-                          bd + ((nh * 4 * SK_B_SLAB + j * 2048) >> 4), idesc, (acc | (uint32_t)j) != 0 ? 1u : 0u);
-              }
+              for (int j = 0; j < SK_AK / 16; ++j)
+                umma_bf16(tmem_base + nh * SK_BNH, desc64(a_lo + (uint32_t)(j * 2), a_hi),
+                          desc64(b_lo + (uint32_t)((j * 2048) >> 4), b_hi), idesc, j == 0 ? acc : 1u);
             }
+            PS_TRACE_ADD(tr_m_is, tis);
             // the tests of the next stages travel while the commits are issued
-            MBAR_PEEK(1, fullb_bar(sb_next), phb_next);
-            if (half == 1) {
-              if (C == 1) { MBAR_PEEK(0, fulla_bar(sa_next), pha_next); } else { MBAR_PEEK_CLUSTER(0, fulla_bar(sa_next), pha_next); }
+            bpeek = ks + 1 < sg.ks1;
+            if (bpeek) {
+              int sbn = qn + myoff;
+              uint32_t phbn = qphn;
+              if (sbn >= SK_B_STAGES) { sbn -= SK_B_STAGES; phbn ^= 1u; }
+              MBAR_PEEK(1, fullb_bar(sbn), phbn);
             }
-            if (issuer) {
-              umma_commit(emptyb_bar(sb));
-              if (half == 1) {
-                // tell every CTA of the cluster (all of them write into this stage) that this CTA is done with it
-#pragma unroll
-                for (int r = 0; r < C; ++r) umma_commit(peer_emptya0[r] + 8u * sa);
-              }
-            }
-            __syncwarp();
-            acc = 1;
-            sb = sb_next;
-            phb = phb_next;
+          } else {
+            issuer = elect_one();
           }
+          PS_TRACE_T0(tco);
+          if (C == 1) { MBAR_PEEK(0, fulla_bar(sa_next), pha_next); } else { MBAR_PEEK_CLUSTER(0, fulla_bar(sa_next), pha_next); }
+          if (issuer) {
+            if (mine) umma_commit(emptyb_bar(sb));
+            // tell every CTA of the cluster (all of them write into this stage) that this warp is done with it
+#pragma unroll
+            for (int r = 0; r < C; ++r) umma_commit(peer_emptya0[r] + 8u * sa);
+          }
+          __syncwarp();
+          PS_TRACE_ADD(tr_m_co, tco);
+          acc = 1;
+          qs = qn;
+          qph = qphn;
           sa = sa_next;
           pha = pha_next;
         }
@@ -505,6 +552,10 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
           if (elect_one()) umma_commit(accfull_bar);
           __syncwarp();
         }
+      }
+      if (warp == 1 && lane == 0) {
+        PS_TRACE_PUT(3, tr_ws); PS_TRACE_PUT(4, tr_wd); PS_TRACE_PUT(5, tr_wa); PS_TRACE_PUT(6, clock64() - tr_sk0);
+        PS_TRACE_PUT(20, tr_m_is); PS_TRACE_PUT(21, tr_m_co);
       }
     }
     __syncwarp();
@@ -530,6 +581,12 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
     int seg_it = 0;
     long long cursor = 0;
     SketchSegment sg;
+    PS_TRACE_DECL(tr_gen);
+    PS_TRACE_DECL(tr_gw);
+    PS_TRACE_DECL(tr_g_ar);
+    PS_TRACE_DECL(tr_dw);
+    PS_TRACE_DECL(tr_dr);
+    PS_TRACE_T0(tr_gl0);
     for (; ok && sketch_next_segment(sc, cl, seg_it, cursor, sg); ++seg) {
       const int tile = sg.tile;
       const long long m0 = (long long)(tile / sc.tiles_n) * SK_BM;
@@ -542,6 +599,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
         const uint32_t pha = (uint32_t)(step / SK_A_STAGES) & 1u;   // and its parity
         // Generate first, into registers: the entries do not depend on the ring, so the wait for
         // the free stage only covers the stores.
+        PS_TRACE_T0(tg0);
         uint4 v[TASKS_PER_THREAD];
         uint32_t off[TASKS_PER_THREAD];
 #pragma unroll
@@ -551,9 +609,13 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
           v[it] = sketch_chunk<DIST>(pk, p, m0 + r, (long long)ks * SK_AK + 8 * c);
           off[it] = (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
         }
+        PS_TRACE_ADD(tr_gen, tg0);
+        PS_TRACE_T0(tgw);
         const bool freed = (C == 1) ? mbar_wait_warp(emptya_bar(sa), pha ^ 1u, abort_flag, p.status)
                                     : mbar_wait_cluster_warp(emptya_bar(sa), pha ^ 1u, abort_flag, p.status);
+        PS_TRACE_ADD(tr_gw, tgw);
         if (!freed) { ok = false; break; }
+        PS_TRACE_T0(tar);
         uint8_t* const stage_ptr = a_ring + sa * SK_A_BYTES;
 #pragma unroll
         for (int it = 0; it < TASKS_PER_THREAD; ++it) *reinterpret_cast<uint4*>(stage_ptr + off[it]) = v[it];
@@ -582,18 +644,24 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
             }
           }
         }
+        PS_TRACE_ADD(tr_g_ar, tar);
       }
       step0 += len;
+      PS_TRACE_T0(tdw);
       ok = ok && mbar_wait_warp(accfull_bar, (uint32_t)seg & 1u, abort_flag, p.status);
+      PS_TRACE_ADD(tr_dw, tdw);
       if (!ok) break;
       tc_fence_after();
+      PS_TRACE_T0(tdr);
       {
         const int q = warp & 3;                 // tensor-memory lane quarter of this warp
         const int cgroup = gw >> 2;             // index among the SK_GEN_WARPS / 4 warps that share the quarter
         float* slot = p.partial + (sg.slot * C + rank) * (long long)SK_TILE_ELEMS;
         float* prow = slot + (long long)(q * 32 + lane) * 4;   // this lane's row, quad-major layout
 #pragma unroll 1
+        const long long n0d = (long long)((tile % sc.tiles_n) * C + (int)rank) * SK_BN;
         for (int c = cgroup; c < SK_BN / 32; c += SK_GEN_WARPS / 4) {   // 32-column chunks, dealt round-robin
+          if (n0d + c * 32 >= p.cols) break;    // columns beyond the result: nothing was accumulated, nothing is read
           uint32_t v[32];
           tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
           tmem_ld_wait();
@@ -605,6 +673,11 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(accempty_bar);
+      PS_TRACE_ADD(tr_dr, tdr);
+    }
+    if (warp == 1 + SK_MMA_WARPS && lane == 0) {
+      PS_TRACE_PUT(8, tr_gen); PS_TRACE_PUT(9, tr_gw); PS_TRACE_PUT(10, clock64() - tr_gl0); PS_TRACE_PUT(18, tr_g_ar);
+      PS_TRACE_PUT(11, tr_dw); PS_TRACE_PUT(12, tr_dr);
     }
   }
   // ---------------------------------------------------------------- teardown
@@ -616,6 +689,7 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
   tc_fence_before();
   if (C == 1) __syncthreads(); else cluster_sync_all();   // nobody leaves while a neighbour may still store or signal here
   if (warp == 1) tmem_dealloc(tmem_base, 512);
+  if (threadIdx.x == 0) PS_TRACE_PUT(0, clock64() - trace_kernel0);
 }
 
 // Layout of a partial tile (128 rows x 512 columns, fp32): column quads are outermost, element
