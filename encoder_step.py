@@ -200,7 +200,14 @@ def main():
     ap.add_argument("--batch", type=int, default=32)
     ap.add_argument("--seq", type=int, default=128)
     ap.add_argument("--fused-qkv", action="store_true", help="one 768 -> 2304 layer (one S, one X_proj) for Q, K, V")
+    # Default 2: in this eager-PyTorch harness the step is bound by the host's enqueue rate (about a thousand small
+    # launches per step), and the side-by-side mode enqueues four more stream operations per pass; the per-layer
+    # benchmark (bench.py), where the GPU is the bound, uses the library's default 0.
+    ap.add_argument("--pass-mode", type=int, default=2, choices=[0, 1, 2],
+                    help="how the library runs a pass: 0 two kernels side by side, 1 one launch, 2 two kernels in turn")
     a = ap.parse_args()
+    import paper_2201_13195_b200 as P
+    P.rmm_set_pass_mode(a.pass_mode)
     cfg = Config(**ROBERTA_BASE, rho=a.rho, dist=a.dist, fused_qkv=a.fused_qkv)
     res = {}
     for kind in ("rmm", "exact"):
@@ -213,7 +220,7 @@ def main():
             "warmup": max(a.warmup, 3), "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "roberta_base_encoder", "layers": cfg.layers, "hidden": cfg.hidden, "ffn": cfg.ffn,
                        "batch": a.batch, "seq": a.seq, "rho": a.rho, "sketch": a.dist, "optimizer": "AdamW (fused)",
-                       "fused_qkv": a.fused_qkv},
+                       "fused_qkv": a.fused_qkv, "pass_mode": a.pass_mode},
             "exact_linear_ms": res["exact"]["ms_per_step"],
             "saved_activation_bytes": {
                 "block_linear_inputs_rmm": res["rmm"]["saved_bytes_block_linear_inputs"],

@@ -130,6 +130,7 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj,
  *      static schedule).  Same results up to the order of the fp32 partial sums; slower on B200 for the Gaussian
  *      sketch (the generation of S does not keep up with two SMs that share every generated entry through the
  *      tensor cores' pair mode), kept as an alternative and for measurements.
+ *   2: the two kernels of mode 0 one after the other on the caller's stream, each on the whole device.
  * Returns RMM_ERR_INVALID_ARG for any other value.
  */
 rmm_status rmm_set_pass_mode(int mode);
@@ -154,14 +155,16 @@ rmm_status rmm_debug_gauss_words(const uint32_t* words, int64_t n, float* out, v
 /*
  * Host-only testing aid (no device needed): the static work schedule of the sketch kernels
  * for a result of `rows` x `cols` contracted over `tokens`, on `max_ctas` CTAs.  CTAs work in
- * clusters of C (4, 2 or 1, whichever divides the number of 512-column blocks); a "tile" is
+ * clusters of C (2 when the result has at least two 512-column blocks, else 1); a "tile" is
  * 128 rows x C 512-column blocks and a "cta" in the records is one cluster.
  *   mode 0: one record (cta, tile, first step, end step, slot) per work segment, in the
  *           order in which each CTA executes them;
  *   mode 1: one record (tile, slot, 0, 0, 0) per partial tile in the order in which the
  *           reduction adds them.
  * Writes at most `cap` records of five int64 to `records` (host memory) and returns the
- * number of records that exist; info[0..4] = tiles, 64-token steps per tile, clusters, slots, C.
+ * number of records that exist; info[0..7] = tiles, 64-token steps per tile, clusters, slots, C, rounds of
+ * whole tiles, full token blocks per remaining tile, width of the last block (0: none, the tiles are cut into
+ * equal blocks only).
  */
 int64_t rmm_debug_sketch_schedule(int64_t rows, int64_t cols, int64_t tokens, int max_ctas, int mode,
                                   int64_t* records, int64_t cap, int64_t* info);

@@ -275,9 +275,10 @@ def rmm_debug_pass_schedule(gemm, sketch, max_pairs=74):
 
 def rmm_debug_sketch_schedule(rows, cols, tokens, max_ctas=148, mode=0):
     """(records, info): the sketch kernels' static schedule as lists of 5-tuples (host only)."""
-    info = (C.c_int64 * 5)()
+    info = (C.c_int64 * 8)()
     n = _lib.rmm_debug_sketch_schedule(rows, cols, tokens, max_ctas, mode, None, 0, C.addressof(info))
     buf = (C.c_int64 * (5 * max(n, 1)))()
     _lib.rmm_debug_sketch_schedule(rows, cols, tokens, max_ctas, mode, C.addressof(buf), n, C.addressof(info))
     recs = [tuple(buf[5 * i + j] for j in range(5)) for i in range(n)]
-    return recs, {"tiles": info[0], "ksteps": info[1], "num_ctas": info[2], "num_slots": info[3], "cluster": info[4]}
+    return recs, {"tiles": info[0], "ksteps": info[1], "num_ctas": info[2], "num_slots": info[3], "cluster": info[4],
+                  "rounds": info[5], "full_blocks": info[6], "w_last": info[7]}

@@ -73,7 +73,8 @@ Workspace workspace_layout(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rm
   if (dt == RMM_DTYPE_BF16) {
     const SketchGeometry gf = sketch_geometry(k, D_in, N), gb = sketch_geometry(k + 1, D_out, N);
     const int tmax = gf.tiles() > gb.tiles() ? gf.tiles() : gb.tiles();
-    off += align_up((size_t)tmax * sizeof(unsigned long long));
+    // completion flags of the partial tiles: one per partial tile and CTA of a cluster (or pair)
+    off += align_up(((size_t)tmax + 2 * tc::SK_MAX_CTAS) * 2 * sizeof(unsigned long long));
     scratch_pass = gf.scratch_bytes() > gb.scratch_bytes() ? gf.scratch_bytes() : gb.scratch_bytes();
   }
   w.g_off = off;
@@ -399,6 +400,15 @@ rmm_status launch_sors_fast(const void* b, void* out, void* ones_out, int64_t k,
   return RMM_OK;
 }
 
+// Tag of a launch: the completion flags of its partial tiles carry it, so that values left in a workspace by
+// earlier launches (or never initialised) read as "not yet".  64 bits from a counter that starts at a
+// time-dependent value: a stale word equals the tag of a later launch with probability 2^-64 per flag.
+unsigned long long next_launch_tag() {
+  static std::atomic<unsigned long long> counter{
+      (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count() * 0x9E3779B97F4A7C15ull};
+  return counter.fetch_add(0x9E3779B97F4A7C15ull) + 1;
+}
+
 rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, int64_t cols, int64_t tokens, float c,
                          int dist, const PhiloxKey& pk, float* partial, int* status, cudaStream_t stream,
                          bool clear_status = false, int clusters_limit = 0) {
@@ -423,7 +433,6 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   int max_clusters = device_state().sketch_clusters[C];
   if (clusters_limit > 0 && clusters_limit < max_clusters) max_clusters = clusters_limit;
   p.sched = tc::make_sketch_schedule(p.rows, cols, tokens, C, max_clusters);
-  const int per_tile = C;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -437,7 +446,11 @@ rmm_status launch_sketch(const void* b, void* out, void* ones_out, int64_t k, in
   cudaError_t le = cudaLaunchKernelEx(&cfg, sketch_kernel_fn(C, dist), tmB, p, pk);
   if (le != cudaSuccess) return RMM_ERR_CUDA;
   note_launches(2);
-  dim3 rgrid((unsigned)(p.sched.tiles() * per_tile), tc::SK_BN / tc::SKR_CHUNK);
+  // The partial tiles are added up by a second, short kernel: measured against a reduction at the end of the sketch
+  // kernel itself (completion flags per partial tile, every warp of the grid taking rows), the separate launch is
+  // 5 us per pass faster on the 4096-token shapes (its blocks start as soon as SMs are free, and the sketch CTAs do
+  // not sit on their SMs while the slowest cluster drains).
+  dim3 rgrid((unsigned)(p.sched.tiles() * C), tc::SK_BN / tc::SKR_CHUNK);
   tc::sketch_reduce_kernel<<<rgrid, tc::SK_BM, 0, stream>>>(p, c, reinterpret_cast<__nv_bfloat16*>(out),
                                                       reinterpret_cast<__nv_bfloat16*>(ones_out));
   return cudaGetLastError() == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
@@ -535,14 +548,6 @@ tc::PassSchedule make_pass_schedule(bool with_gemm, int64_t gM, int64_t gN, int6
   }
   s.gemm_begin[tc::PS_MAX_PAIRS + 1] = acc;
   return s;
-}
-
-// 48-bit tag of a launch: the tickets of the sketch tiles carry it, so that counts left in a workspace by
-// earlier launches (or never initialised) read as zero.
-unsigned long long next_launch_tag() {
-  static std::atomic<unsigned long long> counter{
-      (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count() * 0x9E3779B97F4A7C15ull};
-  return (counter.fetch_add(1) + 1) & ((1ull << 48) - 1);
 }
 
 // One pass: optional dense part C = A B^T (+ bias), A [M][K]; B [N][K] (B_K) or [K][N] (B_MN); optional sketch
@@ -651,7 +656,33 @@ struct PassSplit {
   int sketch_clusters;
 };
 
+PassSplit plan_pass_split_uncached(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens);
+
+// The plan depends on the shape only (and on the device's residency counts, the same for every B200 of a process
+// in practice): the last few shapes are remembered, so that a layer that is called again costs no search.
 PassSplit plan_pass_split(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens) {
+  struct Entry { int64_t key[6]; int dev; PassSplit plan; };
+  static std::mutex mu;
+  static std::vector<Entry> cache;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  const int64_t key[6] = {gM, gN, gK, rows, cols, tokens};
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (const Entry& e : cache)
+      if (e.dev == dev && memcmp(e.key, key, sizeof(key)) == 0) return e.plan;
+  }
+  const PassSplit plan = plan_pass_split_uncached(gM, gN, gK, rows, cols, tokens);
+  std::lock_guard<std::mutex> lock(mu);
+  if (cache.size() >= 64) cache.erase(cache.begin());
+  Entry e;
+  memcpy(e.key, key, sizeof(key));
+  e.dev = dev; e.plan = plan;
+  cache.push_back(e);
+  return plan;
+}
+
+PassSplit plan_pass_split_uncached(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens) {
   PassSplit best = {0, 0};
   const DeviceState& ds = device_state();
   const int C = tc::sketch_cluster_size(cols);
@@ -770,6 +801,7 @@ rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, i
 
   if (dt == RMM_DTYPE_BF16) {
     float* scratch = reinterpret_cast<float*>(ws + w.scratch_off);
+    unsigned long long* tickets = reinterpret_cast<unsigned long long*>(ws + w.ticket_off);
     const size_t scratch_bytes = w.total - w.scratch_off;
     // the first kernel of the call resets the status word (no separate memset on the stream)
     if (dist == RMM_DIST_SORS_HADAMARD && sors_fast_supported(B_proj, D_in, N, scratch_bytes)) {
@@ -788,14 +820,15 @@ rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, i
       PassArgs a;
       if (Y) { a.a = X; a.b = W; a.bias = b; a.c = Y; a.M = N; a.N = D_out; a.K = D_in; a.bmode = tc::B_K; }
       a.data = X; a.out = X_proj; a.k = B_proj; a.cols = D_in; a.tokens = N; a.scale = c; a.dist = (int)dist;
-      return launch_pass(a, pk, scratch, reinterpret_cast<unsigned long long*>(ws + w.ticket_off), status, stream, true);
+      return launch_pass(a, pk, scratch, tickets, status, stream, true);
     }
     if (!Y) {
       ScopedTiming t(RMM_STEP_SKETCH, stream);
       return launch_sketch(X, X_proj, nullptr, B_proj, D_in, N, c, dist, pk, scratch, status, stream, true);
     }
     // Y = X W^T + 1 b^T and X_proj = S^T X: two kernels that share the device and the X stream
-    const PassSplit split = plan_pass_split(N, D_out, D_in, B_proj, D_in, N);
+    const PassSplit split = g_pass_mode.load(std::memory_order_relaxed) == 2 ? PassSplit{0, 0}
+                                                                              : plan_pass_split(N, D_out, D_in, B_proj, D_in, N);
     ScopedTiming t(RMM_STEP_FWD, stream);
     auto gemm = [&](cudaStream_t s_, int pairs) {
       return launch_tc<tc::A_K, tc::B_K>(X, W, Y, b, N, D_out, D_in, 1.0f, status, s_, nullptr, true, pairs);
@@ -840,6 +873,7 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
 
   if (dt == RMM_DTYPE_BF16) {
     float* scratch = reinterpret_cast<float*>(ws + w.scratch_off);
+    unsigned long long* tickets = reinterpret_cast<unsigned long long*>(ws + w.ticket_off);
     const size_t scratch_bytes = w.total - w.scratch_off;
     // the first kernel of the call resets the status word (no separate memset on the stream)
     if (dist == RMM_DIST_SORS_HADAMARD && sors_fast_supported(B_proj, D_out, N, scratch_bytes)) {
@@ -857,7 +891,7 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
       PassArgs a;
       if (dX) { a.a = dY; a.b = W; a.c = dX; a.M = N; a.N = D_in; a.K = D_out; a.bmode = tc::B_MN; }
       a.data = dY; a.out = G; a.ones_out = db; a.k = B_proj; a.cols = D_out; a.tokens = N; a.scale = c; a.dist = (int)dist;
-      st = launch_pass(a, pk, scratch, reinterpret_cast<unsigned long long*>(ws + w.ticket_off), status, stream, true);
+      st = launch_pass(a, pk, scratch, tickets, status, stream, true);
       if (st != RMM_OK) return st;
     } else if (!dX) {
       ScopedTiming t(RMM_STEP_SDY, stream);
@@ -866,7 +900,8 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
     } else {
       // dX = dY W and G = S^T dY (with db = dY^T 1 as the row of ones of S^T): two kernels that share the device and
       // the dY stream
-      const PassSplit split = plan_pass_split(N, D_in, D_out, B_proj + 1, D_out, N);
+      const PassSplit split = g_pass_mode.load(std::memory_order_relaxed) == 2
+                                  ? PassSplit{0, 0} : plan_pass_split(N, D_in, D_out, B_proj + 1, D_out, N);
       ScopedTiming t(RMM_STEP_BWD, stream);
       auto gemm = [&](cudaStream_t s_, int pairs) {
         return launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, status, s_, nullptr, true, pairs);
@@ -945,6 +980,7 @@ int64_t rmm_debug_sketch_schedule(int64_t rows, int64_t cols, int64_t tokens, in
   const tc::SketchSchedule sc = tc::make_sketch_schedule(rows, cols, tokens, C, max_ctas / C > 0 ? max_ctas / C : 1);
   if (info) {
     info[0] = sc.tiles(); info[1] = sc.ksteps; info[2] = sc.num_ctas; info[3] = sc.num_slots(); info[4] = C;
+    info[5] = sc.rounds; info[6] = sc.full_blocks; info[7] = sc.w_last;
   }
   int64_t n = 0;
   auto put = [&](int64_t a, int64_t b, int64_t c, int64_t d, int64_t e) {
@@ -1096,7 +1132,7 @@ int rmm_debug_pass_trace(long long* host_out) {
 #endif
 
 rmm_status rmm_set_pass_mode(int mode) {
-  if (mode != 0 && mode != 1) return RMM_ERR_INVALID_ARG;
+  if (mode < 0 || mode > 2) return RMM_ERR_INVALID_ARG;
   g_pass_mode.store(mode, std::memory_order_relaxed);
   return RMM_OK;
 }

@@ -321,6 +321,42 @@ __device__ long long g_pass_trace[148][PS_TRACE_SLOTS];
 #define PS_TRACE_PUT(slot, value)
 #endif
 
+// ---------------------------------------------------------------- completion flags across CTAs
+// A CTA that has stored a partial result raises its flag: it writes the launch's tag (unique per launch, so that
+// values left by earlier launches, or never written, read as "not yet") with release semantics.  A reader polls
+// the flags it needs with acquire loads.  No atomics: nothing to reset, no contention between the writers.
+__device__ __forceinline__ void flag_raise(unsigned long long* f, unsigned long long tag) {
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(f), "l"(tag) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_acquire_gpu(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+// Bounded wait of a whole warp until the `count` flags f[first], f[first + stride], ... all carry `tag`
+// (lane i polls the flags i, i + 32, ...).  Returns false on abort or when the limit runs out.
+__device__ __forceinline__ bool flags_wait_warp(const unsigned long long* f, long long first, long long stride, int count,
+                                                unsigned long long tag, volatile int* abort_flag, int* status) {
+  const int lane = (int)(threadIdx.x & 31);
+  const long long t0 = clock64();
+  for (uint32_t polls = 0; polls < kWaitLimitPolls; ++polls) {
+    bool mine = true;
+    for (int i = lane; i < count; i += 32) mine = mine && ld_acquire_gpu(f + first + (long long)i * stride) == tag;
+    if (__all_sync(0xffffffffu, mine)) return true;
+    __nanosleep(100);
+    if ((polls & 0xf) == 0xf) {
+      const bool stop = *abort_flag != 0 || clock64() - t0 > kWaitLimitCycles;
+      if (__any_sync(0xffffffffu, stop)) break;
+    }
+  }
+  if (lane == 0 && *abort_flag == 0) {
+    *abort_flag = 1;
+    if (status) atomicExch(status, kStatusTimeout);
+  }
+  __syncwarp();
+  return false;
+}
+
 // ---------------------------------------------------------------- descriptors
 // Shared-memory matrix descriptor, 128-byte swizzle.  Bits: [0,14) start address >> 4,
 // [16,30) leading byte offset >> 4, [32,46) stride byte offset >> 4, [46,48) version = 1,

@@ -88,8 +88,8 @@ struct PassParams {
   int ones_row, slab_map;
   uint32_t sors_mask;
   float* partial;                 // [units][128][cwp] fp32
-  unsigned long long* tickets;    // [sketch tiles]
-  unsigned long long tag;         // 48 bits, unique per launch
+  unsigned long long* tickets;    // [units][2] flags: the CTA has stored its part of the unit's partial tile
+  unsigned long long tag;         // unique per launch
   __nv_bfloat16* sk_out;          // [B_proj][cols]
   __nv_bfloat16* ones_out;        // [cols] or nullptr
   int* status;
@@ -146,42 +146,6 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst_smem, const CUtens
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst_smem), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y), "r"(z)
       : "memory");
-}
-
-// Ticket of a sketch tile: (tag << 16) | arrivals.  A word that carries another tag is left over
-// from an earlier launch (or was never written) and counts as zero arrivals.
-__device__ __forceinline__ void ticket_arrive(unsigned long long* t, unsigned long long tag) {
-  unsigned long long old = *reinterpret_cast<volatile unsigned long long*>(t);
-  for (int tries = 0; tries < (1 << 20); ++tries) {
-    const unsigned long long cnt = ((old >> 16) == tag) ? (old & 0xffffull) : 0ull;
-    const unsigned long long nw = (tag << 16) | (cnt + 1);
-    const unsigned long long prev = atomicCAS(t, old, nw);
-    if (prev == old) return;
-    old = prev;
-  }
-}
-__device__ __forceinline__ unsigned long long ld_acquire_gpu(const unsigned long long* p) {
-  unsigned long long v;
-  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-// Bounded wait until the ticket shows `expected` arrivals of this launch.
-__device__ __forceinline__ bool ticket_wait(const unsigned long long* t, unsigned long long tag, unsigned expected,
-                                            volatile int* abort_flag, int* status) {
-  const unsigned long long want = (tag << 16) | (unsigned long long)expected;
-  if (ld_acquire_gpu(t) == want) return true;
-  const long long t0 = clock64();
-  for (uint32_t polls = 1; polls < kWaitLimitPolls; ++polls) {
-    if (ld_acquire_gpu(t) == want) return true;
-    __nanosleep(200);
-    if ((polls & 0xf) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) break;
-    }
-  }
-  *abort_flag = 1;
-  if (status) atomicExch(status, kStatusTimeout);
-  return false;
 }
 
 #ifndef PS_EXP_GUARD
@@ -624,7 +588,7 @@ pass_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const uint32_t n = atomicAdd(drain_count, 1u);
           if ((n % PS_DRAIN_WARPS) == PS_DRAIN_WARPS - 1) {
             __threadfence();
-            ticket_arrive(p.tickets + t, p.tag);
+            flag_raise(p.tickets + (long long)u * 2 + rank, p.tag);
           }
           mbar_arrive_cluster(skempty_leader);
         }
@@ -710,7 +674,6 @@ pass_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (sk_units > 0) {
     __syncwarp();
     const int total_warps = (int)gridDim.x * PS_WARPS;
-    const unsigned expected = (unsigned)(sc.nb * 2);      // one arrival per CTA and unit
     int checked_tile = -1;
     bool ok = true;
     PS_TRACE_DECL(tr_rw);
@@ -721,11 +684,11 @@ pass_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const long long j = (long long)tm * PS_ROWS + r;
       if (j >= p.rows) continue;
       if (t != checked_tile) {
-        int good = 1;
+        // the flags of both CTAs of every unit (token block) of this tile: units t, t + tiles, ...
         PS_TRACE_T0(tw);
-        if (lane == 0) good = ticket_wait(p.tickets + t, p.tag, expected, abort_flag, p.status) ? 1 : 0;
+        ok = flags_wait_warp(p.tickets, (long long)t * 2, (long long)sk_tiles * 2, sc.nb, p.tag, abort_flag, p.status) &&
+             flags_wait_warp(p.tickets, (long long)t * 2 + 1, (long long)sk_tiles * 2, sc.nb, p.tag, abort_flag, p.status);
         PS_TRACE_ADD(tr_rw, tw);
-        ok = __shfl_sync(0xffffffffu, good, 0) != 0;
         if (!ok) break;
         checked_tile = t;
       }

@@ -126,17 +126,103 @@ CASES = [
 ]
 
 
-@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
-def test_layer_parity_small(case):
-    name, dtype, N, Di, Do, k, dist = case
-    w = R.small_case(name, dtype, N, Di, Do, k, dist, seed=len(name) * 1000003)
-    got = run_layer(w)
+def _check_layer(w, N, Di, Do, k, dist, dtype, got):
     K = contraction_lengths(N, Di, Do, k)
     ref = oracle_layer(w, got["inputs"], gpu_xproj=got["X_proj"])
     assert_parity(got, ref, dtype, K=K, dist=dist)
     # end to end (oracle's own fp64 X_proj in backward)
     ref2 = oracle_layer(w, got["inputs"])
     assert_parity(got, ref2, dtype, names=("dW",), K=K, end_to_end=True, dist=dist)
+
+
+@pytest.fixture
+def pass_mode():
+    """Sets how the library runs a bf16 pass for one test and puts the default back afterwards."""
+    P = _P()
+    yield P.rmm_set_pass_mode
+    P.rmm_set_pass_mode(0)
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+def test_layer_parity_small(case):
+    name, dtype, N, Di, Do, k, dist = case
+    w = R.small_case(name, dtype, N, Di, Do, k, dist, seed=len(name) * 1000003)
+    _check_layer(w, N, Di, Do, k, dist, dtype, run_layer(w))
+
+
+# Shapes chosen for the launch paths they reach, small enough for a full-tensor fp64 comparison.
+PATH_CASES = [
+    # dX is 75 x 4 = 300 tiles of 256 x 256 with a single K block: four and more tiles per CTA pair, both
+    # accumulator buffers reused twice; Y has 75 tiles
+    ("gemm_many_tiles_per_pair", 19200, 1024, 64, 16, R.DIST_RADEMACHER),
+    # forward sketch: 22 row tiles x 4 column groups = 88 tile groups on 74 clusters: a round of whole tiles, then
+    # the remaining tiles cut into token blocks
+    ("sketch_whole_tile_round_and_remainder", 2900, 4096, 64, 2816, R.DIST_GAUSSIAN),
+    # backward sketch: 10 row tiles (1153 rows with the row of ones) x 4 column groups = 40 tile groups on 74
+    # clusters: one full block per tile and a last, narrower block shared tile after tile by the other clusters
+    ("sketch_last_block_line", 4096, 64, 4096, 1152, R.DIST_RADEMACHER),
+]
+
+
+@pytest.mark.parametrize("case", PATH_CASES, ids=[c[0] for c in PATH_CASES])
+def test_layer_parity_launch_paths(case, pass_mode):
+    """Every element of every output against the oracle on shapes that reach the remaining branches of the static
+    schedules, with the two kernels of a pass side by side (default) and one after the other on the whole device
+    (the grid the schedule branches below are stated for)."""
+    P = _P()
+    name, N, Di, Do, k, dist = case
+    w = R.small_case(name, R.DTYPE_BF16, N, Di, Do, k, dist, seed=len(name) * 7919)
+    if name == "sketch_whole_tile_round_and_remainder":
+        _, info = P.rmm_debug_sketch_schedule(k, Di, N, 148)
+        assert info["rounds"] >= 1 and info["tiles"] % info["num_ctas"] != 0
+    if name == "sketch_last_block_line":
+        _, info = P.rmm_debug_sketch_schedule(k + 1, Do, N, 148)
+        assert info["rounds"] == 0 and info["w_last"] > 0
+    if name == "gemm_many_tiles_per_pair":
+        assert -(-N // 256) * -(-Di // 256) >= 4 * 74
+    inputs = R.make_inputs(w)
+    X, W, b, dY = [None if a is None else a.astype(np.float64) for a in inputs]
+    S = O.generate_s(w.seed, N, k, dist, O.STORE_BF16)
+    Y, Xp = O.forward(X, W, b, S)
+    K = contraction_lengths(N, Di, Do, k)
+    for mode in (0, 2):
+        pass_mode(mode)
+        got = run_layer(w, inputs=inputs)
+        dX, dW, db, G = O.backward(dY, W, got["X_proj"], S)      # stage-wise: the GPU's own X_proj
+        ref = {"Y": Y, "X_proj": Xp, "dX": dX, "dW": dW, "db": db, "G": G, "X_proj_used": got["X_proj"]}
+        assert_parity(got, ref, R.DTYPE_BF16, K=K, dist=dist)
+
+
+ONE_LAUNCH_CASES = [c for c in CASES if c[1] == R.DTYPE_BF16 and c[0] in (
+    "tiny_ragged_bf16", "one_row", "multi_tile_ragged_bf16", "multi_tile_ragged_rad", "rho_one_gauss",
+    "k_multiple_of_tile", "sors_below_fast_path", "dx_second_wave")]
+
+
+@pytest.mark.parametrize("case", ONE_LAUNCH_CASES, ids=[c[0] for c in ONE_LAUNCH_CASES])
+def test_layer_parity_one_launch_per_pass(case, pass_mode):
+    """The alternative execution of a pass as a single launch (sketch units and dense tiles of one static schedule,
+    in-kernel reduction of the partial tiles): same gates as the default path."""
+    name, dtype, N, Di, Do, k, dist = case
+    pass_mode(1)
+    w = R.small_case(name, dtype, N, Di, Do, k, dist, seed=len(name) * 1000003)
+    _check_layer(w, N, Di, Do, k, dist, dtype, run_layer(w))
+
+
+@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS])
+def test_one_launch_pass_sketch_bit_exact(dist, pass_mode):
+    """S entry by entry through the one-launch pass kernel (X = selector matrix), several token blocks per tile."""
+    P = _P()
+    pass_mode(1)
+    N, D, k, seed = 16500, 1024, 141, 91
+    rng = np.random.default_rng(seed)
+    tokens = np.sort(rng.choice(N, size=D, replace=False))
+    X = _selector(N, tokens, R.DTYPE_BF16)
+    W = torch.zeros((8, D), dtype=torch.bfloat16, device="cuda")
+    _, Xp = P.rmm_forward(X, W, None, seed, k, dist, want_y=False)
+    torch.cuda.synchronize()
+    Pm = O.generate_p(seed, N, k, dist, O.STORE_BF16)[tokens]
+    want = R.round_to_bf16((Pm.T * np.float32(O.scale(k, dist))).astype(np.float32))
+    assert np.array_equal(Xp.to(torch.float32).cpu().numpy(), want)
 
 
 def test_identity_sketch_is_exact_layer():
@@ -275,4 +361,11 @@ def test_full_size_sampled(name):
 
 @pytest.mark.parametrize("name", ["base_ffn_up_rho0.1", "base_ffn_up_rho0.5", "base_ffn_up_rho0.9"])
 def test_full_size_sampled_other_rho(name):
+    assert _sampled_full_size(name)
+
+
+@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("name", ["base_qkv_rad_rho0.2", "large_ffn_up_rho0.1"])
+def test_full_size_sampled_other_pass_modes(name, mode, pass_mode):
+    pass_mode(mode)
     assert _sampled_full_size(name)
