@@ -173,6 +173,25 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_variance_probe(args, w, P, Xd, dYd):
+    """Times rmm_variance_probe (the variance diagnostics of Section 2.3 on the device) on the workload's X and dY."""
+    import torch
+    pws = torch.empty(P.rmm_variance_probe_workspace_bytes(w.n_tokens, w.d_in, w.d_out), dtype=torch.uint8, device="cuda")
+    out = torch.empty(8, dtype=torch.float64, device="cuda")
+    for _ in range(args.warmup):
+        P.rmm_variance_probe(Xd, dYd, w.b_proj, w.dist, out=out, workspace=pws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        P.rmm_variance_probe(Xd, dYd, w.b_proj, w.dist, out=out, workspace=pws)
+    e1.record()
+    torch.cuda.synchronize()
+    assert P.rmm_last_device_status(pws) == P.RMM_OK
+    print(json.dumps({"metric": "rmm_variance_probe time", "unit": "ms", "value": e0.elapsed_time(e1) / args.steps,
+                      "config": workload_config(w), "values": dict(zip(P.VARIANCE_FIELDS, out.cpu().tolist()))}), flush=True)
+
+
 def workload_config(w):
     touched = (2 * w.n_tokens * (w.d_in + w.d_out) * 2 + 3 * w.d_in * w.d_out + 2 * w.b_proj * (w.d_in + w.d_out)) * w.elem_bytes
     return {"workload": w.name, "n_tokens": w.n_tokens, "d_in": w.d_in, "d_out": w.d_out, "rho": w.rho,
@@ -204,6 +223,17 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(R.WORKLOADS))
+    ap.add_argument("--shape", type=int, nargs=4, metavar=("N", "D_IN", "D_OUT", "B_PROJ"), default=None,
+                    help="an ad-hoc bf16 layer instead of a named workload (small cases for profilers)")
+    ap.add_argument("--dist", default="gaussian", choices=["gaussian", "rademacher", "sors"], help="sketch of --shape")
+    ap.add_argument("--pass-mode", type=int, default=0, choices=[0, 1, 2],
+                    help="0: the two kernels of a pass side by side (default), 1: one launch per pass, 2: one after the other")
+    ap.add_argument("--cycle-trace", action="store_true",
+                    help="with the cycle-accounting build of the library (RMM_LIBRARY=...): print the per-role cycle "
+                         "counters of the last sketch / one-launch kernel to stderr (median and maximum over CTAs)")
+    ap.add_argument("--forward-only", action="store_true", help="steps are forward passes only (for profilers)")
+    ap.add_argument("--variance-probe", action="store_true",
+                    help="time rmm_variance_probe on the workload's X and dY instead of the layer")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -211,7 +241,12 @@ def main():
                     help="wall-clock budget of the whole --impl reference run (sizes its token sample)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    w = R.WORKLOADS[args.workload]
+    if args.shape is not None:
+        n, di, do, k = args.shape
+        dist = {"gaussian": R.DIST_GAUSSIAN, "rademacher": R.DIST_RADEMACHER, "sors": R.DIST_SORS}[args.dist]
+        w = R.Workload(f"shape_{n}_{di}_{do}_k{k}_{args.dist}", R.DTYPE_BF16, n, di, do, k / n, dist, 0, k_fixed=k)
+    else:
+        w = R.WORKLOADS[args.workload]
 
     if args.impl == "reference":
         run_reference(args, w)
@@ -228,6 +263,7 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
     torch.cuda.set_device(local_rank)
+    P.rmm_set_pass_mode(args.pass_mode)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
@@ -244,10 +280,15 @@ def main():
     ws = P.alloc_workspace(N, w.d_in, w.d_out, k, w.dtype)
     stream = torch.cuda.current_stream()
 
+    if args.variance_probe:
+        run_variance_probe(args, w, P, Xd, dYd)
+        return
+
     def step(i):
         seed = w.seed + i          # a fresh S every step (Algorithm 1)
         P.rmm_forward(Xd, Wd, None, seed, k, w.dist, Y=Y, X_proj=Xp, workspace=ws, stream=stream)
-        P.rmm_backward(dYd, Wd, Xp, seed, w.dist, dX=dX, dW=dW, db=db, workspace=ws, stream=stream)
+        if not args.forward_only:
+            P.rmm_backward(dYd, Wd, Xp, seed, w.dist, dX=dX, dW=dW, db=db, workspace=ws, stream=stream)
 
     def barrier():
         if world > 1:
@@ -277,6 +318,15 @@ def main():
     assert P.rmm_last_device_status(ws) == P.RMM_OK
     records = P.rmm_profile_read(min(args.steps, 200) * 6)
     P.rmm_profile_enable(0)
+    if args.cycle_trace and rank == 0:
+        tr = P.rmm_debug_pass_trace()
+        if tr is None:
+            sys.stderr.write("no cycle counters: load the cycle-accounting build with RMM_LIBRARY=...\n")
+        else:
+            for name, v in tr.items():
+                lead, peer = [x for x in v[0::2] if x], [x for x in v[1::2] if x]
+                fmt = lambda a: f"median {int(np.median(a)):9d} max {max(a):9d}" if a else "-"
+                sys.stderr.write(f"{name:22s} even CTAs {fmt(lead)}   odd CTAs {fmt(peer)}\n")
 
     ms_total = max_over_ranks(ms_total, torch.device("cuda", local_rank))
     ms_step = ms_total / args.steps
@@ -292,6 +342,8 @@ def main():
     peaks = load_peaks()
     flops_of = {"y": fl["y"], "sketch": fl["sketch"], "dx": fl["dx"], "sdy": fl["sdy"], "dw": fl["dw"],
                 "fwd": fl["y"] + fl["sketch"], "bwd": fl["dx"] + fl["sdy"]}
+    if "bwd" in per_kernel and "dw" not in per_kernel:
+        flops_of["bwd"] += fl["dw"]          # dW ran inside the backward pass (beside dX, after the sketch)
     for name, d in per_kernel.items():
         if name in flops_of:
             d["tflops"] = flops_of[name] / (d["ms"] * 1e-3) / 1e12
@@ -319,7 +371,7 @@ def main():
 
     # ---- end to end through the host-buffer entry points (pinned host memory)
     e2e = None
-    if rank == 0 or world > 1:
+    if (rank == 0 or world > 1) and args.e2e_steps > 0:
         # E2E_LANES lanes (stream, device staging, workspace, host result buffers) take the steps in turn, so that
         # the host->device copies of one step overlap the device->host copies of the step before it (the two
         # copy directions are separate engines); every step still copies all its inputs in and all its results out.
@@ -388,7 +440,7 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16" if w.dtype == R.DTYPE_BF16 else "f32", "data": "synthetic",
-                "config": workload_config(w), "clocks": clocks, "e2e": e2e,
+                "config": {**workload_config(w), "pass_mode": args.pass_mode}, "clocks": clocks, "e2e": e2e,
                 "gpu_launches": gpu_launches, "roofline": roofline, "cpu_baseline": cpu,
                 "pct_of_tensor_peak": {"burst": 100 * value / world / peaks["bf16_tflops"],
                                        "sustained": 100 * value / world / peaks["bf16_tflops_sustained"],

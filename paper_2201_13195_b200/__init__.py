@@ -8,7 +8,7 @@ no non-CUDA path: using the package without a built library raises ImportError.
 import importlib
 
 
-_SUBMODULES = ("build", "binding", "run_case")
+_SUBMODULES = ("build", "binding")
 
 
 def __getattr__(name):

@@ -10,7 +10,9 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "librmm.so")
+# RMM_LIBRARY names another build of the same library (e.g. the cycle-accounting build made by
+# `python -m paper_2201_13195_b200.build --trace FILE`); by default the in-tree librmm.so is loaded.
+LIB_PATH = os.environ.get("RMM_LIBRARY") or os.path.join(_HERE, "librmm.so")
 
 RMM_OK, RMM_ERR_INVALID_ARG, RMM_ERR_UNSUPPORTED, RMM_ERR_WORKSPACE, RMM_ERR_CUDA, RMM_ERR_TIMEOUT = range(6)
 RMM_DIST_GAUSSIAN, RMM_DIST_RADEMACHER, RMM_DIST_IDENTITY, RMM_DIST_SORS_HADAMARD = 0, 1, 2, 3
@@ -252,6 +254,25 @@ def rmm_debug_gauss_words(words, stream=None):
 def rmm_set_pass_mode(mode: int) -> None:
     """0: the two kernels of a pass side by side (default); 1: one launch per pass."""
     _check(_lib.rmm_set_pass_mode(int(mode)), "rmm_set_pass_mode")
+
+
+TRACE_SLOTS = ("kernel", "producer_wait", "producer_loop", "mma_wait_s", "mma_wait_data", "mma_wait_accumulator",
+               "mma_sketch_loop", "mma_dense_loop", "generator_arithmetic", "generator_wait_stage", "generator_loop",
+               "drain_wait", "drain", "epilogue_loop", "reduction_wait", "reduction", "generator_store", "generator_fence",
+               "generator_handover", "mma_fence", "mma_issue", "mma_commit")
+
+
+def rmm_debug_pass_trace():
+    """Cycle counters of the last sketch or one-launch pass kernel, per CTA: {slot name: [148 values]}.  Only the
+    cycle-accounting build of the library (RMM_LIBRARY) exports them; returns None otherwise."""
+    if not hasattr(_lib, "rmm_debug_pass_trace"):
+        return None
+    buf = (C.c_longlong * (148 * 32))()
+    _lib.rmm_debug_pass_trace.argtypes = [_vp]
+    _lib.rmm_debug_pass_trace.restype = _int
+    if _lib.rmm_debug_pass_trace(C.addressof(buf)) != 0:
+        return None
+    return {name: [int(buf[cta * 32 + i]) for cta in range(148)] for i, name in enumerate(TRACE_SLOTS)}
 
 
 def rmm_layer_launch_count() -> int:

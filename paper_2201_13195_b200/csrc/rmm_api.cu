@@ -656,23 +656,27 @@ struct PassSplit {
   int sketch_clusters;
 };
 
-PassSplit plan_pass_split_uncached(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens);
+PassSplit plan_pass_split_uncached(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens,
+                                   int64_t tail_m, int64_t tail_n, int64_t tail_k);
 
 // The plan depends on the shape only (and on the device's residency counts, the same for every B200 of a process
 // in practice): the last few shapes are remembered, so that a layer that is called again costs no search.
-PassSplit plan_pass_split(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens) {
-  struct Entry { int64_t key[6]; int dev; PassSplit plan; };
+// tail_m x tail_n (contracted over tail_k; 0: none) is a dense product that follows the sketch on its side of the
+// split (dW = G^T X_proj needs G = S^T dY, not dX).
+PassSplit plan_pass_split(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens,
+                          int64_t tail_m = 0, int64_t tail_n = 0, int64_t tail_k = 0) {
+  struct Entry { int64_t key[9]; int dev; PassSplit plan; };
   static std::mutex mu;
   static std::vector<Entry> cache;
   int dev = 0;
   cudaGetDevice(&dev);
-  const int64_t key[6] = {gM, gN, gK, rows, cols, tokens};
+  const int64_t key[9] = {gM, gN, gK, rows, cols, tokens, tail_m, tail_n, tail_k};
   {
     std::lock_guard<std::mutex> lock(mu);
     for (const Entry& e : cache)
       if (e.dev == dev && memcmp(e.key, key, sizeof(key)) == 0) return e.plan;
   }
-  const PassSplit plan = plan_pass_split_uncached(gM, gN, gK, rows, cols, tokens);
+  const PassSplit plan = plan_pass_split_uncached(gM, gN, gK, rows, cols, tokens, tail_m, tail_n, tail_k);
   std::lock_guard<std::mutex> lock(mu);
   if (cache.size() >= 64) cache.erase(cache.begin());
   Entry e;
@@ -682,7 +686,8 @@ PassSplit plan_pass_split(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int6
   return plan;
 }
 
-PassSplit plan_pass_split_uncached(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens) {
+PassSplit plan_pass_split_uncached(int64_t gM, int64_t gN, int64_t gK, int64_t rows, int64_t cols, int64_t tokens,
+                                   int64_t tail_m, int64_t tail_n, int64_t tail_k) {
   PassSplit best = {0, 0};
   const DeviceState& ds = device_state();
   const int C = tc::sketch_cluster_size(cols);
@@ -690,12 +695,17 @@ PassSplit plan_pass_split_uncached(int64_t gM, int64_t gN, int64_t gK, int64_t r
   if (total < 2 || !ds.lanes_ok) return best;
   const long long G = ((gN + tc::BN - 1) / tc::BN) * ((gM + tc::PAIR_M - 1) / tc::PAIR_M);
   const long long num_kb = (gK + tc::BK - 1) / tc::BK;
-  // costs in SM cycles: a dense tile (4 MMAs of 128 cycles per K block, plus fill and epilogue), a 64-token sketch step
-  const long long cg = num_kb * 540 + 3000, cstep = 1460, fixed = 6000;
+  // costs in SM cycles, from the launch lists under profiles/: a dense tile (about 500 cycles per K block of 64, plus
+  // fill and epilogue), a 64-token sketch step
+  const long long cg = num_kb * 500 + 800, cstep = 1460, fixed = 6000;
   auto gemm_cost = [&](int pairs) { return ((G + pairs - 1) / pairs) * cg + fixed; };
+  const long long tail_tiles = tail_m > 0 ? ((tail_n + tc::BN - 1) / tc::BN) * ((tail_m + tc::PAIR_M - 1) / tc::PAIR_M) : 0;
+  const long long tail_cg = ((tail_k + tc::BK - 1) / tc::BK) * 500 + 800;
   auto sketch_cost = [&](int clusters) {
     const tc::SketchSchedule sc = tc::make_sketch_schedule(rows, cols, tokens, C, C == 2 ? clusters : 2 * clusters);
-    return sc.est_steps * cstep + fixed + 9000;    // + the reduction kernel
+    long long t = sc.est_steps * cstep + fixed + 9000;    // + the reduction kernel
+    if (tail_tiles > 0) t += ((tail_tiles + clusters - 1) / clusters) * tail_cg + fixed;
+    return t;
   };
   const long long serial = gemm_cost(total) + sketch_cost(total);
   long long best_cost = serial;
@@ -901,8 +911,8 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
       // dX = dY W and G = S^T dY (with db = dY^T 1 as the row of ones of S^T): two kernels that share the device and
       // the dY stream
       const PassSplit split = g_pass_mode.load(std::memory_order_relaxed) == 2
-                                  ? PassSplit{0, 0} : plan_pass_split(N, D_in, D_out, B_proj + 1, D_out, N);
-      ScopedTiming t(RMM_STEP_BWD, stream);
+                                  ? PassSplit{0, 0}
+                                  : plan_pass_split(N, D_in, D_out, B_proj + 1, D_out, N, D_out, D_in, B_proj);
       auto gemm = [&](cudaStream_t s_, int pairs) {
         return launch_tc<tc::A_K, tc::B_MN>(dY, W, dX, nullptr, N, D_in, D_out, 1.0f, status, s_, nullptr, true, pairs);
       };
@@ -910,11 +920,21 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
         return launch_sketch(dY, G, db, B_proj, D_out, N, c, dist, pk, scratch, status, s_, false, clusters);
       };
       if (split.gemm_pairs == 0) {
+        ScopedTiming t(RMM_STEP_BWD, stream);
         st = gemm(stream, 0);
         if (st == RMM_OK) st = sketch(stream, 0);
       } else {
-        st = fork_join(stream, [&](cudaStream_t side) { return sketch(side, split.sketch_clusters); },
-                       [&](cudaStream_t main_) { return gemm(main_, split.gemm_pairs); });
+        // dW = G^T X_proj follows the sketch on the side stream, on the SMs that the sketch kernel leaves: it needs
+        // G, not dX, so it runs beside the rest of the dX product
+        ScopedTiming t(RMM_STEP_BWD, stream);
+        return fork_join(stream,
+                         [&](cudaStream_t side) {
+                           rmm_status s1 = sketch(side, split.sketch_clusters);
+                           if (s1 != RMM_OK) return s1;
+                           return launch_tc<tc::A_MN, tc::B_MN>(G, X_proj, dW, nullptr, D_out, D_in, B_proj, 1.0f, status, side,
+                                                                nullptr, false, split.sketch_clusters);
+                         },
+                         [&](cudaStream_t main_) { return gemm(main_, split.gemm_pairs); });
       }
       if (st != RMM_OK) return st;
     }

@@ -30,17 +30,23 @@
 //
 // Warp roles: warp 0 TMA producer (B); warps 1-2 MMA issuers, one per 256-column half of the
 // accumulator (warp 1 owns the tensor memory); warps 3..14 generate S tiles, in three groups of
-// four that each own one ring stage, and drain the accumulator.  A ring: 3 stages of 64 tokens;
-// B ring: 5 stages of 32 tokens (the B ring is the latency-critical one: it holds 2.5 K-steps).
-// What limits the kernel: a 64-token step moves 80 KB of operands through shared memory, so the
-// two rings hold about 2.6 steps, less than the round trip MMA completion -> commit -> producer
-// -> (TMA load | stores + bulk copy to the peer) -> MMA issue.  With all generator arithmetic
-// or all B loads removed (experiments) the kernel is less than 10 % faster: neither the ALUs nor
-// L2 nor the tensor pipe (about 70 % busy in steady state) is the bound, the ring depth is.
+// four that each own one ring stage, and drain the accumulator.  A ring: 3 stages of 64 tokens x
+// 128 rows; B ring: 5 stages of 64 tokens x 256 columns, each consumed by one MMA warp (one barrier
+// round per four MMAs).
+// What limits the kernel (cycle counters of the RMM_PASS_TRACE build, 256-step segments): a 64-token
+// step takes about 1400 cycles with the Gaussian sketch against 1024 cycles of tensor work.  The
+// generators need about 930 cycles of arithmetic per step (three groups in turn) plus the hand-over
+// of the stage (stores, proxy fence, count, bulk copy to the peer: 360 cycles), and the MMA warps
+// wait about 450 cycles per step for S^T: the generation of the normals is the bound.  With the
+// Rademacher sketch the generators are idle, but a step takes 1800 cycles: a stage is refilled the
+// moment it is freed, while the tensor pipe reads operands at full rate (96 bytes per cycle of MMA
+// operand reads plus 64 of TMA writes per SM), and the generators' ordinary stores into shared memory
+// then complete slowly: the same hand-over takes 1700 cycles.  The tensor pipe itself runs every
+// operand layout used here at its nominal 8192 FLOP per cycle and SM when fed from resident tiles.
 // Barriers of a CTA: fullA[s] (the group's warps + the bytes copied in by the other CTAs: the
-// stage is complete in this CTA's ring), emptyA[s] (2 C commits: every MMA warp of every CTA of
-// the cluster has consumed the stage, so it may be overwritten everywhere), fullB / emptyB (TMA
-// ring; 2 commits), accfull / accempty.  All waits are bounded.
+// stage is complete in this CTA's ring), emptyA[s] (2 C commits: every MMA warp of every CTA of the
+// cluster has consumed the stage, so it may be overwritten everywhere), fullB / emptyB (TMA
+// ring; one commit, by the warp the stage belongs to), accfull / accempty.  All waits are bounded.
 #pragma once
 #include "sketch_rng.cuh"
 #include "tc_common.cuh"
