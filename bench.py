@@ -28,11 +28,13 @@ import rmm_inputs as R  # noqa: E402
 METRIC = "RMM linear fwd+bwd TFLOP/s (bf16)"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "large_ffn_up_rho0.1"
-# (workload, step) -> (dram__bytes_read.sum per token row of the kernel's input, dram__bytes_write.sum
-# per launch), from an ncu capture of sketch_kernel<2> at 4096 tokens: 33.70 MB read (the dY stream, in
-# proportion to the tokens), 14.68 MB written (fp32 partial tiles that leave L2; their number follows
-# the schedule, not the token count).
-NCU_DRAM_BYTES = {("large_ffn_up_rho0.1", "sdy"): (33.698304e6 / 4096, 14.677504e6)}
+# (workload, step) -> DRAM bytes of the kernels of that pass, from the ncu capture at 4096 tokens summarised in
+# profiles/dram_bytes_per_kernel_n4096_din1024_dout4096_k1638.md: (bytes read per token row, bytes read once, bytes
+# written).  Backward pass: the sketch kernel reads dY once (33.61 MB per 4096 tokens) and so does the dX kernel
+# (33.59 MB; cold caches, the two kernels serialised by ncu: side by side the second reader is served by L2 as far
+# as dY fits); W 8.39 MB, G + X_proj 16.81 MB once; written at full size: dX, G and dW (at 4096 tokens they stay in L2).
+NCU_DRAM_BYTES = {("large_ffn_up_rho0.1", "bwd"): ((33.613312e6 + 33.59e6) / 4096, 8.39e6 + 16.81e6,
+                                                  lambda w: (w.n_tokens * w.d_in + w.b_proj * w.d_out + w.d_in * w.d_out) * 2)}
 
 STEP_ORDER = ("fwd", "bwd", "y", "sketch", "dx", "sdy", "dw", "db")
 E2E_LANES = 3    # streams (each with its own staging buffers and thread) that take the end-to-end steps in turn
@@ -237,7 +239,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--reference-budget-s", type=float, default=90.0,
+    ap.add_argument("--reference-budget-s", type=float, default=300.0,
                     help="wall-clock budget of the whole --impl reference run (sizes its token sample)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -360,14 +362,19 @@ def main():
                 "peak_kind": f"{'burst' if use_burst else 'sustained'} bf16 GEMM, of {peaks['source']}",
                 "frac_of_burst": achieved / peaks["bf16_tflops"],
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
-                "traffic": None, "algorithmic_flops_per_launch": flops_of[dom]}
-    # DRAM bytes per launch of the dominant step, from an ncu capture taken at 4096 tokens; the
-    # reads are the dY stream and grow in proportion to the tokens.
+                "traffic": None, "algorithmic_flops_per_launch": flops_of[dom],
+                "kernel_note": {"fwd": "forward pass: dense kernel (Y) beside sketch kernel (X_proj) + its reduction",
+                                "bwd": "backward pass: dense kernel (dX) beside sketch kernel (S^T dY, db) + reduction + dW kernel"
+                                }.get(dom, dom)}
+    # DRAM bytes of the dominant pass, from an ncu capture taken at 4096 tokens; the token-sized reads grow in
+    # proportion to the tokens.
     ncu_traffic = NCU_DRAM_BYTES.get((w.name, dom))
-    if ncu_traffic is not None:
-        roofline["traffic"] = ncu_traffic[0] * w.n_tokens + ncu_traffic[1]
-        roofline["traffic_note"] = ("dram read+write of sketch_kernel<2,0>: ncu at 4096 tokens, reads scaled by tokens, "
-                                    "writes (partial tiles) as captured")
+    if ncu_traffic is not None and args.pass_mode == 0:
+        roofline["traffic"] = ncu_traffic[0] * w.n_tokens + ncu_traffic[1] + ncu_traffic[2](w)
+        roofline["algorithmic_bytes"] = (w.n_tokens * (w.d_out + w.d_in) + w.d_in * w.d_out * 2 + w.b_proj * (2 * w.d_out + w.d_in)) * 2
+        roofline["traffic_note"] = ("dram read+write of the kernels of the backward pass (dX kernel, sketch kernel, dW kernel): "
+                                    "ncu at 4096 tokens, cold cache per kernel, token-sized reads scaled by the token count, "
+                                    "results counted once")
 
     # ---- end to end through the host-buffer entry points (pinned host memory)
     e2e = None

@@ -5,7 +5,7 @@
 // db = dY^T 1 as one more row of S^T).  pass_kernel does both in one launch: every CTA pair of the
 // grid first works on its share of the sketch, then on its share of the dense tiles, and at the
 // end all warps of the grid add up the partial sketch tiles.  Both kinds of work run on the same
-// pipeline (one TMA ring, one MMA-issuing warp per pair, tcgen05.mma.cta_group::2 throughout), so
+// pipeline (one TMA ring, tcgen05.mma.cta_group::2 throughout), so
 // the dense tiles fill the time that the few, long sketch tiles would leave idle.
 //
 // Dense tiles: as in tc_gemm.cuh (256 x 256 pair tiles, K step 64, two accumulator buffers,
@@ -23,18 +23,23 @@
 // same time walk the same token range, so the token-sized operand is read from HBM once), and
 // every unit leaves one fp32 partial tile.
 //
-// Reduction.  When a warp has stored its part of a partial tile it arrives on the tile's ticket
-// (a tagged counter in the workspace: the tag is unique per launch, so the counters need no
-// reset between launches).  After its last unit every warp of the grid takes rows of the result,
-// waits (bounded) until the row's tile has all its arrivals, adds the partial tiles in block
-// order, applies the scale c = 1/sqrt(B_proj) (Eq. 5), rounds to bf16 and stores.  Sketch units
-// never wait for another pair, so this wait cannot deadlock; it normally finds the count complete.
+// Reduction.  When the warps of a CTA have stored their part of a unit's partial tile, the CTA raises
+// the unit's completion flag: it writes the launch's tag (unique per launch, so flags need no reset
+// between launches; a value left by an earlier launch reads as "not yet").  After its last unit
+// every warp of the grid takes rows of the result, waits (bounded) until the flags of the row's tile
+// are all raised, adds the partial tiles in block order, applies the scale c = 1/sqrt(B_proj)
+// (Eq. 5), rounds to bf16 and stores.  Sketch units never wait for another pair, so this wait cannot
+// deadlock; it normally finds the flags raised.
 //
-// Warp roles per CTA: warp 0 TMA producer; warp 1 tensor-memory owner and (leader CTA) MMA issuer;
-// warps 2-5 epilogue of the dense tiles; warps 6-13 generators of S^T; warps 2-13 drain the sketch
-// accumulators.  Shared memory: ring of 6 stages of 32 KB (dense: 128 x 64 of A and of B; sketch:
-// 32 tokens x nat x 128 data columns), and 32 KB that hold the four 64-token S^T stages while the
-// CTA works on sketch units and the epilogue's store boxes afterwards.  All waits are bounded.
+// Warp roles per CTA: warp 0 TMA producer; warp 1 tensor-memory owner and, in the leader CTA, MMA
+// issuer (dense tiles; accumulators 0 and 1 of the sketch units); warp 14 second MMA issuer of the
+// sketch units (accumulators 2 and 3); warps 2-5 epilogue of the dense tiles; warps 6-13 generators
+// of S^T, four groups of two, group g filling S^T stage g; warps 2-13 drain the sketch accumulators.
+// The generators of the leader CTA arrive on the leader's "S^T stage full" barrier; those of the peer
+// signal it with one asynchronous 4-byte store per stage, counted on the same barrier.  Shared memory:
+// ring of 6 stages of 32 KB (dense: 128 x 64 of A and of B; sketch: 32 tokens x nat x 128 data
+// columns), and 32 KB that hold the four 64-token S^T stages while the CTA works on sketch units and
+// the epilogue's store boxes afterwards.  All waits are bounded.
 #pragma once
 #include "sketch_rng.cuh"
 #include "tc_common.cuh"
