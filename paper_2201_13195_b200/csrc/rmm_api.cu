@@ -79,7 +79,7 @@ Workspace workspace_layout(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rm
   }
   w.g_off = off;
   off = w.g_off + align_up((size_t)k * (size_t)D_out * elem_bytes(dt));
-  int64_t rps = 256;
+  int64_t rps = 32;                       // rows per slice of the fp32 mode's db partial sums: at most 256 slices
   if ((N + rps - 1) / rps > 256) rps = (N + 255) / 256;
   w.db_rows_per_slice = (int)rps;
   w.db_slices = (int)((N + rps - 1) / rps);

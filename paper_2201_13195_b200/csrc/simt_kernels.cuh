@@ -32,7 +32,12 @@ struct SimtGemmArgs {
   uint32_t sors_mask;                  // dist 3: order of the Hadamard matrix - 1
 };
 
-constexpr int SIMT_BM = 64, SIMT_BN = 64, SIMT_BK = 16, SIMT_THREADS = 256;
+// 32 x 64 output tiles (the layer's fp32 shapes are small: with 64 x 64 tiles the 512-token configuration gave
+// 48 to 144 blocks for 148 SMs), 16-deep K slices; the next slice's global loads are issued into registers
+// before the current slice is multiplied, so their latency overlaps the arithmetic.
+constexpr int SIMT_BM = 32, SIMT_BN = 64, SIMT_BK = 16, SIMT_THREADS = 256;
+constexpr int SIMT_A_PER_THREAD = SIMT_BM * SIMT_BK / SIMT_THREADS;   // 2
+constexpr int SIMT_B_PER_THREAD = SIMT_BN * SIMT_BK / SIMT_THREADS;   // 4
 
 template <typename T, bool GEN_A>
 __global__ void __launch_bounds__(SIMT_THREADS)
@@ -41,15 +46,43 @@ simt_gemm_kernel(SimtGemmArgs g, PhiloxKey pk) {
   __shared__ float Bs[SIMT_BK][SIMT_BN + 4];
   const int tid = threadIdx.x;
   const int64_t m0 = (int64_t)blockIdx.y * SIMT_BM, n0 = (int64_t)blockIdx.x * SIMT_BN;
-  const int tx = tid & 15, ty = tid >> 4;   // 16 x 16 threads, 4 x 4 outputs each
-  float acc[4][4] = {};
+  const int tx = tid & 15, ty = tid >> 4;   // 16 x 16 threads, 2 x 4 outputs each
+  float acc[2][4] = {};
   const T* A = reinterpret_cast<const T*>(g.A);
   const T* B = reinterpret_cast<const T*>(g.B);
 
+  // element e of a slice of A / B -> (row in tile, k in slice); the orientation is chosen so that consecutive
+  // threads walk the unit-stride index
+  auto a_coord = [&](int e, int& mm, int& kk) {
+    if (g.a_sk == 1) { kk = e % SIMT_BK; mm = e / SIMT_BK; } else { mm = e % SIMT_BM; kk = e / SIMT_BM; }
+  };
+  auto b_coord = [&](int e, int& nn, int& kk) {
+    if (g.b_sk == 1) { kk = e % SIMT_BK; nn = e / SIMT_BK; } else { nn = e % SIMT_BN; kk = e / SIMT_BN; }
+  };
+  float ra[SIMT_A_PER_THREAD], rb[SIMT_B_PER_THREAD];
+  auto fetch = [&](int64_t k0) {
+    if (!GEN_A) {
+#pragma unroll
+      for (int i = 0; i < SIMT_A_PER_THREAD; ++i) {
+        int mm, kk;
+        a_coord(tid + i * SIMT_THREADS, mm, kk);
+        const int64_t m = m0 + mm, k = k0 + kk;
+        ra[i] = (m < g.M && k < g.K) ? to_f32<T>(A[m * g.a_sm + k * g.a_sk]) : 0.0f;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < SIMT_B_PER_THREAD; ++i) {
+      int nn, kk;
+      b_coord(tid + i * SIMT_THREADS, nn, kk);
+      const int64_t n = n0 + nn, k = k0 + kk;
+      rb[i] = (n < g.N && k < g.K) ? to_f32<T>(B[n * g.b_sn + k * g.b_sk]) : 0.0f;
+    }
+  };
+  fetch(0);
   for (int64_t k0 = 0; k0 < g.K; k0 += SIMT_BK) {
     if (GEN_A) {
-      // 64 sketch columns x 16 tokens: 128 tasks of 8 tokens each.
-      if (tid < 128) {
+      // 32 sketch columns x 16 tokens: 64 tasks of 8 tokens each.
+      if (tid < 2 * SIMT_BM) {
         const int r = tid >> 1, h = tid & 1;
         const int64_t j = m0 + r, n8 = k0 + 8 * h;
         float z[8];
@@ -77,30 +110,30 @@ simt_gemm_kernel(SimtGemmArgs g, PhiloxKey pk) {
         for (int i = 0; i < 8; ++i) As[8 * h + i][r] = (j < g.M && n8 + i < g.K) ? z[i] : 0.0f;
       }
     } else {
-      for (int e = tid; e < SIMT_BM * SIMT_BK; e += SIMT_THREADS) {
-        // orientation chosen so that consecutive threads walk the unit-stride index
+#pragma unroll
+      for (int i = 0; i < SIMT_A_PER_THREAD; ++i) {
         int mm, kk;
-        if (g.a_sk == 1) { kk = e % SIMT_BK; mm = e / SIMT_BK; } else { mm = e % SIMT_BM; kk = e / SIMT_BM; }
-        const int64_t m = m0 + mm, k = k0 + kk;
-        As[kk][mm] = (m < g.M && k < g.K) ? to_f32<T>(A[m * g.a_sm + k * g.a_sk]) : 0.0f;
+        a_coord(tid + i * SIMT_THREADS, mm, kk);
+        As[kk][mm] = ra[i];
       }
     }
-    for (int e = tid; e < SIMT_BN * SIMT_BK; e += SIMT_THREADS) {
+#pragma unroll
+    for (int i = 0; i < SIMT_B_PER_THREAD; ++i) {
       int nn, kk;
-      if (g.b_sk == 1) { kk = e % SIMT_BK; nn = e / SIMT_BK; } else { nn = e % SIMT_BN; kk = e / SIMT_BN; }
-      const int64_t n = n0 + nn, k = k0 + kk;
-      Bs[kk][nn] = (n < g.N && k < g.K) ? to_f32<T>(B[n * g.b_sn + k * g.b_sk]) : 0.0f;
+      b_coord(tid + i * SIMT_THREADS, nn, kk);
+      Bs[kk][nn] = rb[i];
     }
     __syncthreads();
+    if (k0 + SIMT_BK < g.K) fetch(k0 + SIMT_BK);      // in flight while this slice is multiplied
 #pragma unroll
     for (int kk = 0; kk < SIMT_BK; ++kk) {
-      float a[4], b[4];
+      float a[2], b[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+      for (int i = 0; i < 2; ++i) a[i] = As[kk][ty * 2 + i];
 #pragma unroll
       for (int i = 0; i < 4; ++i) b[i] = Bs[kk][tx * 4 + i];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < 2; ++i)
 #pragma unroll
         for (int jn = 0; jn < 4; ++jn) acc[i][jn] = fmaf(a[i], b[jn], acc[i][jn]);
     }
@@ -109,8 +142,8 @@ simt_gemm_kernel(SimtGemmArgs g, PhiloxKey pk) {
   T* C = reinterpret_cast<T*>(g.C);
   const T* bias = reinterpret_cast<const T*>(g.bias);
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int64_t m = m0 + ty * 4 + i;
+  for (int i = 0; i < 2; ++i) {
+    const int64_t m = m0 + ty * 2 + i;
     if (m >= g.M) continue;
 #pragma unroll
     for (int jn = 0; jn < 4; ++jn) {
