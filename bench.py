@@ -56,7 +56,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index, period=0.001):
         super().__init__(daemon=True)
         self.index, self.period = index, period
-        self.samples, self.reasons = [], set()
+        self.samples, self.reasons, self.power = [], set(), []
         self.stop_flag = threading.Event()
         self.max_mhz = None
         self.ok = False
@@ -82,6 +82,7 @@ class ClockSampler(threading.Thread):
         while not self.stop_flag.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
                 mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
                 for n, bit in names.items():
                     if mask & bit:
@@ -94,7 +95,8 @@ class ClockSampler(threading.Thread):
         if not self.ok or not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
         return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w": float(np.median(self.power)) if self.power else None}
 
 
 def physical_gpu_index(local_index):

@@ -123,6 +123,11 @@ CASES = [
     # dX has 38 x 2 = 76 tiles of 256 x 256: more than the 74 CTA pairs, so two pairs take a second tile
     # (both accumulator buffers in use), with ragged last rows: 9700 = 37 * 256 + 228
     ("dx_second_wave", R.DTYPE_BF16, 9700, 512, 64, 16, R.DIST_RADEMACHER),
+    # the RoBERTa-base widths: 768 = one and a half 512-column blocks (the cluster's fourth 256-column half is empty),
+    # 2304 = four and a half (odd block count: the last cluster's second CTA only generates its half of S^T)
+    ("widths_768_2304", R.DTYPE_BF16, 320, 768, 2304, 140, R.DIST_GAUSSIAN),
+    # a ragged last 256-column half: 1160 = 4 * 256 + 136
+    ("ragged_column_half", R.DTYPE_BF16, 200, 1160, 648, 90, R.DIST_RADEMACHER),
 ]
 
 
