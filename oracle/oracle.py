@@ -13,7 +13,7 @@ import numpy as np
 
 from . import build as _build
 
-DIST_GAUSSIAN, DIST_RADEMACHER, DIST_IDENTITY, DIST_SORS = 0, 1, 2, 3
+DIST_GAUSSIAN, DIST_RADEMACHER, DIST_IDENTITY, DIST_SORS, DIST_DCT = 0, 1, 2, 3, 4
 STORE_BF16, STORE_F32 = 0, 1
 
 _lib = C.CDLL(_build.build())

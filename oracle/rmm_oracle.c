@@ -22,7 +22,8 @@
  * independent implementation; the Gaussian transform against fp64 Box-Muller over
  * all 2^16 radius and angle inputs; brute-force numpy loops on tiny shapes; S = I
  * reproducing the exact gradient; Monte-Carlo unbiasedness and variance; the
- * paper's worked 2x2 example for the two variance estimators.
+ * paper's worked 2x2 example for the two variance estimators; the structured
+ * sketches against scipy's Hadamard and DCT-II matrices.
  */
 #include <math.h>
 #include <stdint.h>
@@ -36,6 +37,7 @@
 #define ORACLE_DIST_RADEMACHER 1
 #define ORACLE_DIST_IDENTITY 2
 #define ORACLE_DIST_SORS 3
+#define ORACLE_DIST_DCT 4
 #define ORACLE_STORE_BF16 0
 #define ORACLE_STORE_F32 1
 
@@ -203,6 +205,47 @@ void oracle_generate_p_cols(uint64_t seed, int64_t N, int64_t k, int64_t j0, int
         for (uint64_t b = (uint64_t)n & col; b != 0; b >>= 1) ones += (int)(b & 1u);
         const float h = (ones & 1) ? -1.0f : 1.0f;
         out[n * w + (j - j0)] = d_neg ? -h : h;
+      }
+    }
+    return;
+  }
+  if (dist == ORACLE_DIST_DCT) {
+    /* Subsampled DCT-II with random signs (Section 3.5 compares DCT sketches, Section 2.1 names the SORS
+     * family; the construction is defined here).  L = smallest power of two >= N; the orthonormal DCT-II
+     * matrix of order L has rows C[0][n] = sqrt(1/L), C[r][n] = sqrt(2/L) cos(pi (2n+1) r / (2L)).
+     * P[n][j] = d_n * sqrt(L) * C[r_j][n], with d_n and r_j drawn exactly as for the Hadamard variant
+     * (counters (n>>7,0,0,2) and (j,0,0,3)): 1 for r_j = 0, else sqrt(2) cos(...), where the cosine is
+     * evaluated in fp32: m = (2n+1) r mod 4L (exact integers), quadrant q = m / L, x = (m mod L) / L in
+     * [0,1), and cos(pi/2 (q + x)) = c, -s, -c, s for q = 0..3 with s = x * S(x^2), c = C(x^2), S and C the
+     * cubics of the Gaussian transform's angle step (Horner, fmaf). */
+    uint64_t L = 1;
+    int logL = 0;
+    while (L < (uint64_t)N) { L <<= 1; ++logL; }
+    const float inv_L = bits_f32((uint32_t)(127 - logL) << 23);   /* 2^-logL, exact */
+    const float SQRT2 = 0x1.6a09e6p+0f;
+    for (int64_t j = j0; j < j1; ++j) {
+      uint32_t cj[4] = {(uint32_t)j, 0u, 0u, 3u}, rj[4];
+      oracle_philox4x32_10(cj, key, rj);
+      const uint64_t r = (uint64_t)rj[0] % L;
+      for (int64_t n = 0; n < N; ++n) {
+        uint32_t cn[4] = {(uint32_t)(n >> 7), 0u, 0u, 2u}, rn[4];
+        oracle_philox4x32_10(cn, key, rn);
+        const int t = (int)(n & 127);
+        const int d_neg = (int)((rn[t >> 5] >> (t & 31)) & 1u);
+        float g = 1.0f;
+        if (r != 0) {
+          const uint64_t m = ((2u * (uint64_t)n + 1u) * r) & (4u * L - 1u);
+          const int q = (int)(m >> logL);
+          const float x = (float)(uint32_t)(m & (L - 1u)) * inv_L;
+          const float z = x * x;
+          const float sp = fmaf(fmaf(fmaf(SIN_C[3], z, SIN_C[2]), z, SIN_C[1]), z, SIN_C[0]);
+          const float sn = x * sp;
+          const float cs = fmaf(fmaf(fmaf(COS_C[3], z, COS_C[2]), z, COS_C[1]), z, COS_C[0]);
+          const float v = (q == 0) ? cs : (q == 1) ? -sn : (q == 2) ? -cs : sn;
+          g = SQRT2 * v;
+        }
+        if (storage == ORACLE_STORE_BF16) g = oracle_bf16_round(g);
+        out[n * w + (j - j0)] = d_neg ? -g : g;
       }
     }
     return;

@@ -160,6 +160,39 @@ def test_sors_is_sign_flipped_hadamard_columns():
     assert np.allclose(H @ H.T, np.eye(32), atol=1e-12)
 
 
+def test_dct_is_sign_flipped_scaled_dct2_rows():
+    """P[n][j] = d_n * sqrt(L) * C[r_j][n] with C the orthonormal DCT-II matrix of order L (scipy's, an independent
+    library), d_n and r_j from the independent Philox transcription; N not a power of two takes the first N
+    columns of the next order.  The fp32 cosine (quadrant reduction + two cubics) stays within 2e-5 of the exact one."""
+    from scipy.fft import dct
+    for seed, N, k in ((3, 64, 9), (0xABCDEF0123456789, 300, 7), (7, 1, 2), (11, 129, 4), (5, 1000, 3)):
+        L = 1
+        while L < N:
+            L *= 2
+        Cm = dct(np.eye(L), type=2, norm="ortho", axis=0)          # Cm[r][n]
+        assert np.allclose(Cm @ Cm.T, np.eye(L), atol=1e-12)       # the matrix the sketch subsamples is orthonormal
+        key = [seed & M32, seed >> 32]
+        P = O.generate_p(seed, N, k, O.DIST_DCT, O.STORE_F32).astype(np.float64)
+        d = np.array([-1.0 if (_philox_python([n >> 7, 0, 0, 2], key)[(n & 127) >> 5] >> (n & 31)) & 1 else 1.0
+                      for n in range(N)])
+        for j in range(k):
+            r = _philox_python([j, 0, 0, 3], key)[0] % L
+            want = d * math.sqrt(L) * Cm[r, :N]
+            assert np.abs(P[:, j] - want).max() < 2e-5, (seed, N, j, r)
+        Pb = O.generate_p(seed, N, k, O.DIST_DCT, O.STORE_BF16)
+        assert np.array_equal(Pb, R.round_to_bf16(P.astype(np.float32)))
+        S = O.generate_s(seed, N, k, O.DIST_DCT, O.STORE_F32)
+        assert np.array_equal(S, P * float(np.float32(1) / np.sqrt(np.float32(k))))
+    # a column with r_j = 0 is the constant row of the DCT: entries d_n exactly
+    seed, N = 0, 8
+    key = [seed & M32, seed >> 32]
+    js = [j for j in range(4000) if _philox_python([j, 0, 0, 3], key)[0] % 8 == 0][:3]
+    assert js
+    for j in js:
+        col = O.generate_p(seed, N, j + 1, O.DIST_DCT, O.STORE_F32, j, j + 1)[:, 0]
+        assert set(np.unique(np.abs(col))) == {1.0}
+
+
 def test_identity_matrix():
     assert np.array_equal(O.generate_s(1, 6, 6, O.DIST_IDENTITY, O.STORE_BF16), np.eye(6))
 
@@ -232,22 +265,24 @@ def test_identity_sketch_reproduces_exact_gradient():
 
 
 # --------------------------------------------------------------- statistical properties
-@pytest.mark.parametrize("dist", [O.DIST_GAUSSIAN, O.DIST_RADEMACHER, O.DIST_SORS])
+@pytest.mark.parametrize("dist", [O.DIST_GAUSSIAN, O.DIST_RADEMACHER, O.DIST_SORS, O.DIST_DCT])
 def test_unbiasedness_of_s_st(dist):
-    N, k, T = 16, 8, 4000
+    N, k, T = (13 if dist == O.DIST_DCT else 16), 8, 4000      # DCT: a token count that is not a power of two
     acc = np.zeros((N, N))
     for seed in range(T):
         S = O.generate_s(seed, N, k, dist, O.STORE_F32)
         acc += S @ S.T
     M = acc / T
     off = M - np.diag(np.diag(M))
-    sd_diag = math.sqrt((2.0 if dist == O.DIST_GAUSSIAN else 0.0) / (k * T)) + 1e-6
+    # variance of one diagonal term: 2 for normals, 0 for +-1 entries, at most 1/2 for 2 cos^2 - 1 = cos(2 theta)
+    sd_diag = math.sqrt({O.DIST_GAUSSIAN: 2.0, O.DIST_DCT: 1.0}.get(dist, 0.0) / (k * T)) + 1e-6
     assert np.abs(np.diag(M) - 1.0).max() < 4.5 * sd_diag
     assert np.abs(off).max() < 4.5 * math.sqrt(1.0 / (k * T))
 
 
-def test_sors_gradient_is_unbiased():
-    """E_S[dW_rmm] = dW for the subsampled Hadamard sketch (token count not a power of two)."""
+@pytest.mark.parametrize("dist", [O.DIST_SORS, O.DIST_DCT])
+def test_sors_gradient_is_unbiased(dist):
+    """E_S[dW_rmm] = dW for the subsampled Hadamard and DCT sketches (token count not a power of two)."""
     rng = np.random.default_rng(5)
     N, Din, Dout, k, T = 6, 4, 3, 3, 20000
     X = rng.standard_normal((N, Din))
@@ -256,7 +291,7 @@ def test_sors_gradient_is_unbiased():
     dW_star = O.exact_dw(dY, X)
     tot, sq = np.zeros_like(dW_star), np.zeros_like(dW_star)
     for seed in range(T):
-        S = O.generate_s(500 + seed, N, k, O.DIST_SORS, O.STORE_F32)
+        S = O.generate_s(500 + seed, N, k, dist, O.STORE_F32)
         _, Xp = O.forward(X, W, None, S, want_y=False)
         _, dW, _, _ = O.backward(dY, W, Xp, S, want_dx=False, want_db=False)
         tot += dW
