@@ -199,7 +199,7 @@ def run_variance_probe(args, w, P, Xd, dYd):
 def workload_config(w):
     touched = (2 * w.n_tokens * (w.d_in + w.d_out) * 2 + 3 * w.d_in * w.d_out + 2 * w.b_proj * (w.d_in + w.d_out)) * w.elem_bytes
     return {"workload": w.name, "n_tokens": w.n_tokens, "d_in": w.d_in, "d_out": w.d_out, "rho": w.rho,
-            "b_proj": w.b_proj, "sketch": ("gaussian", "rademacher", "identity", "sors_hadamard")[w.dist], "seed": w.seed,
+            "b_proj": w.b_proj, "sketch": ("gaussian", "rademacher", "identity", "sors_hadamard", "sors_dct")[w.dist], "seed": w.seed,
             "l2": f"inputs larger than L2: about {touched / 1e6:.0f} MB of tensors touched per step, no flush"}
 
 
@@ -229,7 +229,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(R.WORKLOADS))
     ap.add_argument("--shape", type=int, nargs=4, metavar=("N", "D_IN", "D_OUT", "B_PROJ"), default=None,
                     help="an ad-hoc bf16 layer instead of a named workload (small cases for profilers)")
-    ap.add_argument("--dist", default="gaussian", choices=["gaussian", "rademacher", "sors"], help="sketch of --shape")
+    ap.add_argument("--dist", default="gaussian", choices=["gaussian", "rademacher", "sors", "dct"], help="sketch of --shape")
     ap.add_argument("--pass-mode", type=int, default=0, choices=[0, 1, 2],
                     help="0: the two kernels of a pass side by side (default), 1: one launch per pass, 2: one after the other")
     ap.add_argument("--cycle-trace", action="store_true",
@@ -247,7 +247,7 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.shape is not None:
         n, di, do, k = args.shape
-        dist = {"gaussian": R.DIST_GAUSSIAN, "rademacher": R.DIST_RADEMACHER, "sors": R.DIST_SORS}[args.dist]
+        dist = {"gaussian": R.DIST_GAUSSIAN, "rademacher": R.DIST_RADEMACHER, "sors": R.DIST_SORS, "dct": R.DIST_DCT}[args.dist]
         w = R.Workload(f"shape_{n}_{di}_{do}_k{k}_{args.dist}", R.DTYPE_BF16, n, di, do, k / n, dist, 0, k_fixed=k)
     else:
         w = R.WORKLOADS[args.workload]

@@ -196,7 +196,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--rho", type=float, default=0.2)
-    ap.add_argument("--dist", default="gaussian", choices=["gaussian", "rademacher", "sors"])
+    ap.add_argument("--dist", default="gaussian", choices=["gaussian", "rademacher", "sors", "dct"])
     ap.add_argument("--batch", type=int, default=32)
     ap.add_argument("--seq", type=int, default=128)
     ap.add_argument("--fused-qkv", action="store_true", help="one 768 -> 2304 layer (one S, one X_proj) for Q, K, V")

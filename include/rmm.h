@@ -50,6 +50,13 @@
  *                       applied by a two-level Walsh-Hadamard transform over the token index
  *                       (O(N D log N)); otherwise by the same dense contraction as the other
  *                       distributions.  S is the same matrix either way;
+ *   RMM_DIST_SORS_DCT   subsampled DCT-II matrix with random signs (Section 3.5 and Table 4 compare DCT
+ *                       sketches; the construction is this library's): with L, d_n and r_j as above and C the
+ *                       orthonormal DCT-II matrix of order L, P[n][j] = d_n * sqrt(L) * C[r_j][n], i.e. d_n for
+ *                       r_j = 0 and d_n * sqrt(2) cos(pi (2n+1) r_j / (2L)) otherwise, the cosine evaluated by
+ *                       a fixed fp32 sequence (exact integer quadrant reduction, two cubic polynomials with
+ *                       fused multiply-adds).  E[S S^T] = I exactly up to that sequence's error of 2e-5.
+ *                       Applied by the dense contraction kernels;
  *   RMM_DIST_IDENTITY   S = I (needs B_proj == N; c = 1): the case in which the
  *                       layer reduces to the exact linear layer; meant for tests.
  * In bf16 mode P is rounded to bfloat16 (nearest even) before it is used.
@@ -77,7 +84,8 @@ typedef enum {
   RMM_DIST_GAUSSIAN = 0,
   RMM_DIST_RADEMACHER = 1,
   RMM_DIST_IDENTITY = 2,
-  RMM_DIST_SORS_HADAMARD = 3
+  RMM_DIST_SORS_HADAMARD = 3,
+  RMM_DIST_SORS_DCT = 4
 } rmm_dist;
 typedef enum { RMM_DTYPE_BF16 = 0, RMM_DTYPE_F32 = 1 } rmm_dtype;
 

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("RMM_LIBRARY") or os.path.join(_HERE, "librmm.so")
 
 RMM_OK, RMM_ERR_INVALID_ARG, RMM_ERR_UNSUPPORTED, RMM_ERR_WORKSPACE, RMM_ERR_CUDA, RMM_ERR_TIMEOUT = range(6)
-RMM_DIST_GAUSSIAN, RMM_DIST_RADEMACHER, RMM_DIST_IDENTITY, RMM_DIST_SORS_HADAMARD = 0, 1, 2, 3
+RMM_DIST_GAUSSIAN, RMM_DIST_RADEMACHER, RMM_DIST_IDENTITY, RMM_DIST_SORS_HADAMARD, RMM_DIST_SORS_DCT = 0, 1, 2, 3, 4
 RMM_DTYPE_BF16, RMM_DTYPE_F32 = 0, 1
 
 EXPORTS = ("rmm_workspace_bytes", "rmm_forward", "rmm_backward", "rmm_debug_generate_s",

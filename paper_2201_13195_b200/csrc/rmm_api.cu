@@ -125,24 +125,29 @@ bool allow_big_smem(K kernel, int bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
+constexpr int kNumDists = 5;     // rmm_dist values 0..4
+
 // The sketch kernel for a cluster size (1 or 2) and a distribution (rmm_dist value).
 typedef void (*SketchKernelFn)(const CUtensorMap, tc::SketchParams, PhiloxKey);
 SketchKernelFn sketch_kernel_fn(int c, int dist) {
-  static const SketchKernelFn table[2][4] = {
-      {tc::sketch_kernel<1, 0>, tc::sketch_kernel<1, 1>, tc::sketch_kernel<1, 2>, tc::sketch_kernel<1, 3>},
-      {tc::sketch_kernel<2, 0>, tc::sketch_kernel<2, 1>, tc::sketch_kernel<2, 2>, tc::sketch_kernel<2, 3>}};
-  return table[c == 2 ? 1 : 0][dist & 3];
+  static const SketchKernelFn table[2][kNumDists] = {
+      {tc::sketch_kernel<1, 0>, tc::sketch_kernel<1, 1>, tc::sketch_kernel<1, 2>, tc::sketch_kernel<1, 3>,
+       tc::sketch_kernel<1, 4>},
+      {tc::sketch_kernel<2, 0>, tc::sketch_kernel<2, 1>, tc::sketch_kernel<2, 2>, tc::sketch_kernel<2, 3>,
+       tc::sketch_kernel<2, 4>}};
+  return table[c == 2 ? 1 : 0][dist >= 0 && dist < kNumDists ? dist : 0];
 }
 
 // The pass kernel for an operand mode of the dense part (B_K: Y = X W^T, B_MN: dX = dY W) and a distribution.
 typedef void (*PassKernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, tc::PassParams,
                              PhiloxKey);
 PassKernelFn pass_kernel_fn(int bmode, int dist) {
-  static const PassKernelFn table[2][4] = {
-      {tc::pass_kernel<tc::B_K, 0>, tc::pass_kernel<tc::B_K, 1>, tc::pass_kernel<tc::B_K, 2>, tc::pass_kernel<tc::B_K, 3>},
+  static const PassKernelFn table[2][kNumDists] = {
+      {tc::pass_kernel<tc::B_K, 0>, tc::pass_kernel<tc::B_K, 1>, tc::pass_kernel<tc::B_K, 2>, tc::pass_kernel<tc::B_K, 3>,
+       tc::pass_kernel<tc::B_K, 4>},
       {tc::pass_kernel<tc::B_MN, 0>, tc::pass_kernel<tc::B_MN, 1>, tc::pass_kernel<tc::B_MN, 2>,
-       tc::pass_kernel<tc::B_MN, 3>}};
-  return table[bmode == tc::B_MN ? 1 : 0][dist & 3];
+       tc::pass_kernel<tc::B_MN, 3>, tc::pass_kernel<tc::B_MN, 4>}};
+  return table[bmode == tc::B_MN ? 1 : 0][dist >= 0 && dist < kNumDists ? dist : 0];
 }
 
 // How many clusters of `c` CTAs of kernel `k` can be resident on the device at once.
@@ -184,9 +189,9 @@ void init_device_state(DeviceState& st, int dev) {
   a &= allow_big_smem(tc::gemm_kernel<tc::A_K, tc::B_MN>, tc::GEMM_SMEM_BYTES);
   a &= allow_big_smem(tc::gemm_kernel<tc::A_MN, tc::B_MN>, tc::GEMM_SMEM_BYTES);
   for (int c = 1; c <= 2; ++c)
-    for (int d = 0; d < 4; ++d) a &= allow_big_smem(sketch_kernel_fn(c, d), tc::SK_SMEM_BYTES);
+    for (int d = 0; d < kNumDists; ++d) a &= allow_big_smem(sketch_kernel_fn(c, d), tc::SK_SMEM_BYTES);
   for (int bm = 0; bm < 2; ++bm)
-    for (int d = 0; d < 4; ++d) a &= allow_big_smem(pass_kernel_fn(bm, d), tc::PS_SMEM_BYTES);
+    for (int d = 0; d < kNumDists; ++d) a &= allow_big_smem(pass_kernel_fn(bm, d), tc::PS_SMEM_BYTES);
   if (a) {
     a &= query_clusters(tc::pass_kernel<tc::B_K, 0>, 2, &st.pass_pairs, tc::PS_THREADS, tc::PS_SMEM_BYTES);
     if (st.pass_pairs > tc::PS_MAX_PAIRS) st.pass_pairs = tc::PS_MAX_PAIRS;
@@ -769,10 +774,11 @@ rmm_status check_common(int64_t N, int64_t D_in, int64_t D_out, int64_t k, rmm_d
   if (N < 1 || D_in < 1 || D_out < 1 || k < 1 || k > N) return RMM_ERR_INVALID_ARG;
   if (N > (int64_t)1 << 31 || D_in > (int64_t)1 << 30 || D_out > (int64_t)1 << 30) return RMM_ERR_INVALID_ARG;
   if (dist != RMM_DIST_GAUSSIAN && dist != RMM_DIST_RADEMACHER && dist != RMM_DIST_IDENTITY &&
-      dist != RMM_DIST_SORS_HADAMARD)
+      dist != RMM_DIST_SORS_HADAMARD && dist != RMM_DIST_SORS_DCT)
     return RMM_ERR_INVALID_ARG;
   if (dt != RMM_DTYPE_BF16 && dt != RMM_DTYPE_F32) return RMM_ERR_INVALID_ARG;
   if (dist == RMM_DIST_IDENTITY && k != N) return RMM_ERR_INVALID_ARG;
+  if (dist == RMM_DIST_SORS_DCT && N > ((int64_t)1 << 30)) return RMM_ERR_UNSUPPORTED;   // its index arithmetic is 32-bit
   if (dt == RMM_DTYPE_BF16 && (D_in % 8 != 0 || D_out % 8 != 0)) return RMM_ERR_UNSUPPORTED;
   return RMM_OK;
 }
@@ -968,10 +974,11 @@ rmm_status rmm_debug_generate_s(uint64_t seed, int64_t N, int64_t B_proj, rmm_di
                                 void* cuda_stream) {
   if (N < 1 || B_proj < 1 || B_proj > N || !S_out) return RMM_ERR_INVALID_ARG;
   if (dist != RMM_DIST_GAUSSIAN && dist != RMM_DIST_RADEMACHER && dist != RMM_DIST_IDENTITY &&
-      dist != RMM_DIST_SORS_HADAMARD)
+      dist != RMM_DIST_SORS_HADAMARD && dist != RMM_DIST_SORS_DCT)
     return RMM_ERR_INVALID_ARG;
   if (dt != RMM_DTYPE_BF16 && dt != RMM_DTYPE_F32) return RMM_ERR_INVALID_ARG;
   if (dist == RMM_DIST_IDENTITY && B_proj != N) return RMM_ERR_INVALID_ARG;
+  if (dist == RMM_DIST_SORS_DCT && N > ((int64_t)1 << 30)) return RMM_ERR_UNSUPPORTED;
   if (!device_state().ok) return RMM_ERR_CUDA;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   const PhiloxKey pk = make_philox_key(seed);
@@ -1089,7 +1096,7 @@ rmm_status rmm_variance_probe(const void* X, const void* dY, int64_t N, int64_t 
   rmm_status st = check_common(N, D_in, D_out, B_proj, dist, dt);
   if (st != RMM_OK) return st;
   if (dt != RMM_DTYPE_BF16) return RMM_ERR_UNSUPPORTED;
-  if (dist == RMM_DIST_SORS_HADAMARD) return RMM_ERR_UNSUPPORTED;   // no closed form for its variance here
+  if (dist == RMM_DIST_SORS_HADAMARD || dist == RMM_DIST_SORS_DCT) return RMM_ERR_UNSUPPORTED;   // no closed form here
   if (!X || !dY || !out) return RMM_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(dY) || !aligned16(out) || !aligned16(dW_exact)) return RMM_ERR_INVALID_ARG;
   const ProbeWorkspace w = probe_layout(N, D_in, D_out);

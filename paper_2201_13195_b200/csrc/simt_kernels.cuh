@@ -102,6 +102,12 @@ simt_gemm_kernel(SimtGemmArgs g, PhiloxKey pk) {
           const uint32_t bits = sors_sign_bits_8(pk, (uint32_t)n8, (uint32_t)j, g.sors_mask);
 #pragma unroll
           for (int i = 0; i < 8; ++i) z[i] = ((bits >> i) & 1u) ? -1.0f : 1.0f;
+        } else if (g.dist == 4) {
+          dct_8(pk, (uint32_t)n8, (uint32_t)j, g.sors_mask, z);
+          if (sizeof(T) == 2) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) z[i] = __bfloat162float(__float2bfloat16_rn(z[i]));
+          }
         } else {
 #pragma unroll
           for (int i = 0; i < 8; ++i) z[i] = (n8 + i == j) ? 1.0f : 0.0f;

@@ -312,6 +312,8 @@ __device__ __forceinline__ uint4 sketch_chunk(const PhiloxKey& pk, const SketchP
     v = rademacher_8_bf16(word, (t & 31) >> 3);
   } else if (DIST == 3) {
     v = rademacher_8_bf16(sors_sign_bits_8(pk, (uint32_t)tok8, (uint32_t)j, p.sors_mask), 0);
+  } else if (DIST == 4) {
+    v = dct_8_bf16(pk, (uint32_t)tok8, (uint32_t)j, p.sors_mask);
   } else {
     const long long d = j - tok8;
     uint32_t q0 = 0, q1 = 0, q2 = 0, q3 = 0;

@@ -13,7 +13,7 @@ import torch
 from . import binding as P
 
 _DIST = {"gaussian": P.RMM_DIST_GAUSSIAN, "rademacher": P.RMM_DIST_RADEMACHER, "identity": P.RMM_DIST_IDENTITY,
-         "sors": P.RMM_DIST_SORS_HADAMARD}
+         "sors": P.RMM_DIST_SORS_HADAMARD, "dct": P.RMM_DIST_SORS_DCT}
 
 
 def bproj_from_rho(n_tokens: int, rho: float) -> int:

@@ -14,7 +14,7 @@ from dataclasses import dataclass
 
 import numpy as np
 
-DIST_GAUSSIAN, DIST_RADEMACHER, DIST_IDENTITY, DIST_SORS = 0, 1, 2, 3
+DIST_GAUSSIAN, DIST_RADEMACHER, DIST_IDENTITY, DIST_SORS, DIST_DCT = 0, 1, 2, 3, 4
 DTYPE_BF16, DTYPE_F32 = 0, 1
 
 
@@ -88,6 +88,8 @@ WORKLOADS = {w.name: w for w in [
     # the RoBERTa-large shape with the subsampled-Hadamard sketch (in bf16 mode applied by the two-level Walsh-Hadamard
     # transform; the dense contraction with the same S only outside Hadamard orders 128 .. 16384)
     _w("large_ffn_up_sors_rho0.1", DTYPE_BF16, 16384, 1024, 4096, 0.1, DIST_SORS, 11),
+    # the RoBERTa-large shape with the subsampled-DCT sketch (dense contraction with generated cosines)
+    _w("large_ffn_up_dct_rho0.1", DTYPE_BF16, 16384, 1024, 4096, 0.1, DIST_DCT, 12),
     # diagnostic: the RoBERTa-large shape with the cheap sketch distribution (isolates the cost of the normals)
     _w("large_ffn_up_rad_rho0.1", DTYPE_BF16, 16384, 1024, 4096, 0.1, DIST_RADEMACHER, 9),
 ]}

@@ -21,7 +21,7 @@ def _P():
 
 # ------------------------------------------------------------------ S bit-exact
 @pytest.mark.parametrize("dtype", [R.DTYPE_BF16, R.DTYPE_F32])
-@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS])
+@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS, R.DIST_DCT])
 @pytest.mark.parametrize("N,k,seed", [(37, 5, 0), (300, 130, 0xDEADBEEF12345678), (1024, 64, 3)])
 def test_sketch_dump_bit_exact(dtype, dist, N, k, seed):
     P = _P()
@@ -43,7 +43,7 @@ def test_gaussian_transform_bit_exact_on_all_radius_and_angle_inputs():
 
 
 @pytest.mark.parametrize("dtype", [R.DTYPE_BF16, R.DTYPE_F32])
-@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS])
+@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS, R.DIST_DCT])
 def test_production_kernel_sketch_bit_exact(dtype, dist):
     """X = I makes X_proj = c * P^T: the sketch kernel's own S, entry by entry."""
     P = _P()
@@ -77,7 +77,7 @@ WIDE_S_CASES = [
 ]
 
 
-@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS])
+@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS, R.DIST_DCT])
 @pytest.mark.parametrize("case", WIDE_S_CASES, ids=[c[0] for c in WIDE_S_CASES])
 def test_production_kernel_sketch_bit_exact_wide(case, dist):
     """S entry by entry on the launch shapes of the RoBERTa layers: results wider than one 512-column block
@@ -117,6 +117,9 @@ CASES = [
     ("k_multiple_of_tile", R.DTYPE_BF16, 512, 128, 256, 256, R.DIST_GAUSSIAN),
     ("sors_ragged_bf16", R.DTYPE_BF16, 389, 264, 520, 77, R.DIST_SORS),
     ("sors_ragged_f32", R.DTYPE_F32, 150, 70, 130, 66, R.DIST_SORS),
+    ("dct_ragged_bf16", R.DTYPE_BF16, 389, 264, 520, 77, R.DIST_DCT),
+    ("dct_ragged_f32", R.DTYPE_F32, 150, 70, 130, 66, R.DIST_DCT),
+    ("dct_widths_768_2304", R.DTYPE_BF16, 320, 768, 2304, 140, R.DIST_DCT),
     ("sors_below_fast_path", R.DTYPE_BF16, 37, 24, 40, 5, R.DIST_SORS),          # Hadamard order 64: dense kernel
     ("sors_one_block", R.DTYPE_BF16, 128, 64, 72, 128, R.DIST_SORS),             # order 128: one block, no second level
     ("sors_many_blocks", R.DTYPE_BF16, 2100, 136, 200, 300, R.DIST_SORS),        # order 4096: 32 blocks, last ones empty
@@ -200,7 +203,7 @@ def test_layer_parity_launch_paths(case, pass_mode):
 
 ONE_LAUNCH_CASES = [c for c in CASES if c[1] == R.DTYPE_BF16 and c[0] in (
     "tiny_ragged_bf16", "one_row", "multi_tile_ragged_bf16", "multi_tile_ragged_rad", "rho_one_gauss",
-    "k_multiple_of_tile", "sors_below_fast_path", "dx_second_wave")]
+    "k_multiple_of_tile", "sors_below_fast_path", "dx_second_wave", "dct_ragged_bf16")]
 
 
 @pytest.mark.parametrize("case", ONE_LAUNCH_CASES, ids=[c[0] for c in ONE_LAUNCH_CASES])
@@ -213,7 +216,7 @@ def test_layer_parity_one_launch_per_pass(case, pass_mode):
     _check_layer(w, N, Di, Do, k, dist, dtype, run_layer(w))
 
 
-@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS])
+@pytest.mark.parametrize("dist", [R.DIST_GAUSSIAN, R.DIST_RADEMACHER, R.DIST_SORS, R.DIST_DCT])
 def test_one_launch_pass_sketch_bit_exact(dist, pass_mode):
     """S entry by entry through the one-launch pass kernel (X = selector matrix), several token blocks per tile."""
     P = _P()
@@ -359,7 +362,7 @@ def _sampled_full_size(name):
 
 @pytest.mark.parametrize("name", ["base_ffn_up_rho0.2", "base_ffn_down_rad_rho0.2", "base_qkv_rad_rho0.2",
                                   "large_ffn_up_rho0.1", "large_ffn_down_rho0.1", "large_ffn_up_k1663_aligned",
-                                  "large_ffn_up_sors_rho0.1"])
+                                  "large_ffn_up_sors_rho0.1", "large_ffn_up_dct_rho0.1"])
 def test_full_size_sampled(name):
     assert _sampled_full_size(name)
 
