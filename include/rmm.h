@@ -14,9 +14,15 @@
  *
  * General conventions
  *   - Every tensor pointer is a DEVICE pointer owned by the caller, row-major,
- *     contiguous, 16-byte aligned.  The library allocates no device memory, keeps no
- *     state between calls, never synchronises, and enqueues work only on the CUDA
- *     stream that is passed in (a cudaStream_t cast to void*, NULL = default stream).
+ *     contiguous, 16-byte aligned.  The library allocates no device memory and never
+ *     synchronises.  To the caller all work is ordered on the CUDA stream that is passed in
+ *     (a cudaStream_t cast to void*, NULL = default stream); in the default pass mode part
+ *     of a bf16 pass is queued on a stream of the library's own that forks from and joins
+ *     that stream through events (rmm_set_pass_mode).  What the library keeps between
+ *     calls, per process: per device the kernels' attributes, eight such side streams with
+ *     two events each (created at the first call made with that device current) and the
+ *     address of the fixed scratch of rmm_bias_grad_static; the last 64 pass plans by
+ *     shape; a launch counter.  Results never depend on any of it.
  *   - Outputs are overwritten, never accumulated into.
  *   - dtype RMM_DTYPE_BF16: tensors are bfloat16, contractions run on the tensor
  *     cores with fp32 accumulation; D_in and D_out must be multiples of 8.
@@ -92,7 +98,8 @@ typedef enum { RMM_DTYPE_BF16 = 0, RMM_DTYPE_F32 = 1 } rmm_dtype;
 /*
  * Bytes of scratch device memory that rmm_forward / rmm_backward need for these
  * sizes (the larger of the two).  The scratch holds the intermediate G = S^T dY
- * (B_proj x D_out), partial sums, and a status word.  Returns 0 for invalid sizes.
+ * (B_proj x D_out), fp32 partial tiles of the sketches with their completion flags, and a
+ * status word; it need not be initialised.  Returns 0 for invalid sizes.
  * The same workspace may be reused by later calls on the same stream; calls that may
  * overlap on the device need separate workspaces.
  */
