@@ -449,7 +449,7 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16" if w.dtype == R.DTYPE_BF16 else "f32", "data": "synthetic",
-                "config": {**workload_config(w), "pass_mode": args.pass_mode}, "clocks": clocks, "e2e": e2e,
+                "config": workload_config(w), "pass_mode": args.pass_mode, "clocks": clocks, "e2e": e2e,
                 "gpu_launches": gpu_launches, "roofline": roofline, "cpu_baseline": cpu,
                 "pct_of_tensor_peak": {"burst": 100 * value / world / peaks["bf16_tflops"],
                                        "sustained": 100 * value / world / peaks["bf16_tflops_sustained"],
