@@ -701,8 +701,9 @@ PassSplit plan_pass_split_uncached(int64_t gM, int64_t gN, int64_t gK, int64_t r
   const long long G = ((gN + tc::BN - 1) / tc::BN) * ((gM + tc::PAIR_M - 1) / tc::PAIR_M);
   const long long num_kb = (gK + tc::BK - 1) / tc::BK;
   // costs in SM cycles, from the launch lists under profiles/: a dense tile (about 500 cycles per K block of 64, plus
-  // fill and epilogue), a 64-token sketch step
-  const long long cg = num_kb * 500 + 800, cstep = 1460, fixed = 6000;
+  // fill and epilogue), a 64-token sketch step (1415 cycles measured in steady state; 1300 here splits the 4096-token
+  // shapes best and makes no difference on the 16384-token ones: 1300 / 1460 / 1600 / 1750 were timed back to back)
+  const long long cg = num_kb * 500 + 800, cstep = 1300, fixed = 6000;
   auto gemm_cost = [&](int pairs) { return ((G + pairs - 1) / pairs) * cg + fixed; };
   const long long tail_tiles = tail_m > 0 ? ((tail_n + tc::BN - 1) / tc::BN) * ((tail_m + tc::PAIR_M - 1) / tc::PAIR_M) : 0;
   const long long tail_cg = ((tail_k + tc::BK - 1) / tc::BK) * 500 + 800;
