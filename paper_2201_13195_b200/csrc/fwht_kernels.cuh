@@ -31,11 +31,11 @@ struct SorsGroups {
 
 // One block: r_j for every sketch column, counted and scattered by rb.  The order inside a group
 // depends on the order of the atomics; every entry is written out independently, so it does not
-// affect the result.
-__global__ void __launch_bounds__(1024)
-sors_group_kernel(PhiloxKey pk, int64_t k, uint32_t mask, SorsGroups g, int* status, int clear_status) {
+// affect the result.  Run by the first block of the first stage-1 launch of a sketch (stage 2, which reads the
+// groups, is a later launch on the same stream): the block is the first to be scheduled, and the few
+// microseconds it spends here are over long before the other blocks of the launch are.
+__device__ __forceinline__ void sors_group_block(const PhiloxKey& pk, int64_t k, uint32_t mask, SorsGroups g) {
   __shared__ int count[128], start[129], fill[128];
-  if (clear_status && threadIdx.x == 0) *status = 0;
   if (threadIdx.x < 128) { count[threadIdx.x] = 0; fill[threadIdx.x] = 0; }
   __syncthreads();
   for (int64_t j = threadIdx.x; j < k; j += blockDim.x) {
@@ -59,6 +59,7 @@ sors_group_kernel(PhiloxKey pk, int64_t k, uint32_t mask, SorsGroups g, int* sta
     const int pos = start[rb] + atomicAdd(&fill[rb], 1);
     g.entries[pos] = make_int2((int)j, (int)(r >> 7));
   }
+  __syncthreads();
 }
 
 // The 128-point Walsh-Hadamard transform of a [128 rows][64 columns] tile, rows = 16 g + i.
@@ -89,14 +90,19 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// Stage 1.  grid = (column slabs of 64, A blocks of 128 tokens).  B is [N][ldb] bf16 (this launch
+// Stage 1.  grid = (column slabs of 64, A blocks of 128 tokens); block (0, 0) also builds the column groups.  B is [N][ldb] bf16 (this launch
 // covers `width` columns starting at B); T is [A * 128][ldt] bf16; colsum (nullable) is [A][ldt] fp32.
 __global__ void __launch_bounds__(FW_THREADS)
 fwht_stage1_kernel(const __nv_bfloat16* __restrict__ B, int64_t ldb, int64_t N, int width, PhiloxKey pk,
-                   __nv_bfloat16* __restrict__ T, int64_t ldt, float* __restrict__ colsum) {
+                   __nv_bfloat16* __restrict__ T, int64_t ldt, float* __restrict__ colsum, SorsGroups groups, int64_t k,
+                   uint32_t mask, int* status, int clear_status) {
   __shared__ float2 tile[FW_ROWS][FW_COLS / 2];
   __shared__ float2 part[FW_THREADS / 32][FW_COLS / 2];
   const int tid = threadIdx.x, w = tid >> 5, lane = tid & 31;
+  if (blockIdx.x == 0 && blockIdx.y == 0) {
+    if (clear_status && tid == 0) *status = 0;
+    if (groups.offsets != nullptr) sors_group_block(pk, k, mask, groups);   // only in the first launch of a sketch
+  }
   const int c0 = blockIdx.x * FW_COLS, a = blockIdx.y;
   const int col = c0 + 2 * lane;
   const bool in_cols = col < width;                       // width is a multiple of 8: a column pair is all in or all out

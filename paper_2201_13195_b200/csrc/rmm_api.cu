@@ -385,17 +385,17 @@ rmm_status launch_sors_fast(const void* b, void* out, void* ones_out, int64_t k,
   g.entries = reinterpret_cast<int2*>(base + plan.entries_off);
   float* colsum = reinterpret_cast<float*>(base + plan.colsum_off);
   __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(base + plan.t_off);
-  sors_group_kernel<<<1, 1024, 0, stream>>>(pk, k, mask, g, status, clear_status ? 1 : 0);
-  note_launches(1);
-  if (cudaGetLastError() != cudaSuccess) return RMM_ERR_CUDA;
   const __nv_bfloat16* B = reinterpret_cast<const __nv_bfloat16*>(b);
   __nv_bfloat16* O = reinterpret_cast<__nv_bfloat16*>(out);
   __nv_bfloat16* ones = reinterpret_cast<__nv_bfloat16*>(ones_out);
   for (int64_t c0 = 0; c0 < cols; c0 += wslab) {
     const int width = (int)(cols - c0 < wslab ? cols - c0 : wslab);
     const unsigned slabs = (unsigned)((width + FW_COLS - 1) / FW_COLS);
+    SorsGroups build = g;                                   // the first launch also builds the column groups
+    if (c0 != 0) { build.offsets = nullptr; build.entries = nullptr; }
     fwht_stage1_kernel<<<dim3(slabs, (unsigned)A), FW_THREADS, 0, stream>>>(B + c0, cols, tokens, width, pk, T, wslab,
-                                                                           ones ? colsum : nullptr);
+                                                                           ones ? colsum : nullptr, build, k, mask, status,
+                                                                           (clear_status && c0 == 0) ? 1 : 0);
     if (cudaGetLastError() != cudaSuccess) return RMM_ERR_CUDA;
     note_launches(2);
     fwht_stage2_kernel<<<dim3(slabs, FW_ROWS), FW_THREADS, 0, stream>>>(T, wslab, A, width, g, c, O + c0, cols,

@@ -666,7 +666,6 @@ sketch_kernel(const __grid_constant__ CUtensorMap tmB, SketchParams p, PhiloxKey
         const int cgroup = gw >> 2;             // index among the SK_GEN_WARPS / 4 warps that share the quarter
         float* slot = p.partial + (sg.slot * C + rank) * (long long)SK_TILE_ELEMS;
         float* prow = slot + (long long)(q * 32 + lane) * 4;   // this lane's row, quad-major layout
-#pragma unroll 1
         const long long n0d = (long long)((tile % sc.tiles_n) * C + (int)rank) * SK_BN;
         for (int c = cgroup; c < SK_BN / 32; c += SK_GEN_WARPS / 4) {   // 32-column chunks, dealt round-robin
           if (n0d + c * 32 >= p.cols) break;    // columns beyond the result: nothing was accumulated, nothing is read

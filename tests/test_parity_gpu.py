@@ -123,6 +123,7 @@ CASES = [
     ("sors_below_fast_path", R.DTYPE_BF16, 37, 24, 40, 5, R.DIST_SORS),          # Hadamard order 64: dense kernel
     ("sors_one_block", R.DTYPE_BF16, 128, 64, 72, 128, R.DIST_SORS),             # order 128: one block, no second level
     ("sors_many_blocks", R.DTYPE_BF16, 2100, 136, 200, 300, R.DIST_SORS),        # order 4096: 32 blocks, last ones empty
+    ("sors_wide", R.DTYPE_BF16, 300, 2200, 2312, 40, R.DIST_SORS),                # 35 and 37 column slabs of 64, the last one ragged
     # dX has 38 x 2 = 76 tiles of 256 x 256: more than the 74 CTA pairs, so two pairs take a second tile
     # (both accumulator buffers in use), with ragged last rows: 9700 = 37 * 256 + 228
     ("dx_second_wave", R.DTYPE_BF16, 9700, 512, 64, 16, R.DIST_RADEMACHER),
