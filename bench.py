@@ -281,7 +281,7 @@ def main():
     dX = torch.empty((N, w.d_in), dtype=td, device="cuda")
     dW = torch.empty((w.d_out, w.d_in), dtype=td, device="cuda")
     db = torch.empty((w.d_out,), dtype=td, device="cuda")
-    ws = P.alloc_workspace(N, w.d_in, w.d_out, k, w.dtype)
+    ws = P.alloc_workspace(N, w.d_in, w.d_out, k, w.dtype, dist=w.dist)
     stream = torch.cuda.current_stream()
 
     if args.variance_probe:
@@ -393,7 +393,7 @@ def main():
                   "hd": [torch.empty_like(a, device="cpu").pin_memory() for a in (dX, dW, db)],
                   "dev_in": torch.empty(nb, dtype=torch.uint8, device="cuda"),
                   "dev_out": torch.empty(nb, dtype=torch.uint8, device="cuda"),
-                  "ws": ws if li == 0 else P.alloc_workspace(N, w.d_in, w.d_out, k, w.dtype)}
+                  "ws": ws if li == 0 else P.alloc_workspace(N, w.d_in, w.d_out, k, w.dtype, dist=w.dist)}
             lanes.append(ln)
 
         def e2e_step(i):

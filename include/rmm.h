@@ -106,6 +106,17 @@ typedef enum { RMM_DTYPE_BF16 = 0, RMM_DTYPE_F32 = 1 } rmm_dtype;
 size_t rmm_workspace_bytes(int64_t N, int64_t D_in, int64_t D_out, int64_t B_proj, rmm_dtype dt);
 
 /*
+ * The workspace size with which calls that use sketch `dist` run fastest; never less than
+ * rmm_workspace_bytes(), and equal to it for every distribution but RMM_DIST_SORS_HADAMARD in bf16
+ * mode with at most 16384 tokens.  There the fast transform (Section 2.1: structured sketches have a
+ * fast matrix-by-vector product) keeps an intermediate of L x D bf16 values (L = the Hadamard order,
+ * D = the wider of D_in and D_out) in the workspace; with less room it takes the columns in
+ * several rounds of launches.  Any workspace of at least rmm_workspace_bytes() bytes is valid for
+ * every call; the calls use all of the workspace_bytes they are given.
+ */
+size_t rmm_workspace_bytes_for(int64_t N, int64_t D_in, int64_t D_out, int64_t B_proj, rmm_dtype dt, rmm_dist dist);
+
+/*
  * Algorithm 1, FORWARD (Eq. 1 and X_proj = S^T X, Section 2.1).
  *   in : X [N, D_in], W [D_out, D_in], b [D_out] or NULL (no bias)
  *   out: Y [N, D_out] = X W^T + 1 b^T ;  X_proj [B_proj, D_in] = S^T X

@@ -18,7 +18,7 @@ RMM_OK, RMM_ERR_INVALID_ARG, RMM_ERR_UNSUPPORTED, RMM_ERR_WORKSPACE, RMM_ERR_CUD
 RMM_DIST_GAUSSIAN, RMM_DIST_RADEMACHER, RMM_DIST_IDENTITY, RMM_DIST_SORS_HADAMARD, RMM_DIST_SORS_DCT = 0, 1, 2, 3, 4
 RMM_DTYPE_BF16, RMM_DTYPE_F32 = 0, 1
 
-EXPORTS = ("rmm_workspace_bytes", "rmm_forward", "rmm_backward", "rmm_debug_generate_s",
+EXPORTS = ("rmm_workspace_bytes", "rmm_workspace_bytes_for", "rmm_forward", "rmm_backward", "rmm_debug_generate_s",
            "rmm_last_device_status", "rmm_status_string", "rmm_host_staging_bytes",
            "rmm_forward_host", "rmm_backward_host", "rmm_profile_enable", "rmm_profile_read",
            "rmm_bias_grad_static", "rmm_debug_gauss_words", "rmm_debug_sketch_schedule",
@@ -34,6 +34,8 @@ _lib = C.CDLL(LIB_PATH)
 _i64, _vp, _u64, _int, _sz = C.c_int64, C.c_void_p, C.c_uint64, C.c_int, C.c_size_t
 _lib.rmm_workspace_bytes.argtypes = [_i64, _i64, _i64, _i64, _int]
 _lib.rmm_workspace_bytes.restype = _sz
+_lib.rmm_workspace_bytes_for.argtypes = [_i64, _i64, _i64, _i64, _int, _int]
+_lib.rmm_workspace_bytes_for.restype = _sz
 _lib.rmm_forward.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _int, _int, _vp, _vp, _vp, _sz, _vp]
 _lib.rmm_forward.restype = _int
 _lib.rmm_backward.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _u64, _i64, _int, _int, _vp, _vp, _vp, _vp, _sz, _vp]
@@ -108,8 +110,15 @@ def rmm_workspace_bytes(N, D_in, D_out, B_proj, dt) -> int:
     return int(_lib.rmm_workspace_bytes(N, D_in, D_out, B_proj, dt))
 
 
-def alloc_workspace(N, D_in, D_out, B_proj, dt, device="cuda"):
-    return torch.empty(rmm_workspace_bytes(N, D_in, D_out, B_proj, dt), dtype=torch.uint8, device=device)
+def rmm_workspace_bytes_for(N, D_in, D_out, B_proj, dt, dist) -> int:
+    return int(_lib.rmm_workspace_bytes_for(N, D_in, D_out, B_proj, dt, dist))
+
+
+def alloc_workspace(N, D_in, D_out, B_proj, dt, device="cuda", dist=None):
+    """A workspace of the smallest valid size, or (with `dist`) of the size that suits that sketch best."""
+    nbytes = rmm_workspace_bytes(N, D_in, D_out, B_proj, dt) if dist is None else \
+        rmm_workspace_bytes_for(N, D_in, D_out, B_proj, dt, dist)
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
 
 
 def rmm_forward(X, W, b, seed, B_proj, dist, Y=None, X_proj=None, workspace=None, stream=None, want_y=True):

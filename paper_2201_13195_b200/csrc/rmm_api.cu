@@ -367,6 +367,14 @@ bool sors_fast_plan(int64_t k, int64_t cols, int64_t tokens, size_t scratch_byte
   }
   return true;
 }
+// Scratch with which the fast path takes all `cols` columns in one round (0 outside the fast path).
+size_t sors_fast_full_scratch(int64_t k, int64_t cols, int64_t tokens) {
+  const int64_t L = (int64_t)sors_mask_for(tokens) + 1;
+  if (L < FW_ROWS || L > (int64_t)FW_ROWS * FW_ROWS) return 0;
+  const int64_t cols64 = (cols + FW_COLS - 1) / FW_COLS * FW_COLS;
+  const size_t off = align_up(129 * sizeof(int)) + align_up((size_t)k * sizeof(int2));
+  return off + align_up((size_t)(L / FW_ROWS) * (size_t)cols64 * sizeof(float)) + (size_t)L * (size_t)cols64 * 2 + 4 * kAlign;
+}
 bool sors_fast_supported(int64_t k, int64_t cols, int64_t tokens, size_t scratch_bytes) {
   return sors_fast_plan(k, cols, tokens, scratch_bytes, nullptr);
 }
@@ -800,6 +808,15 @@ size_t rmm_workspace_bytes(int64_t N, int64_t D_in, int64_t D_out, int64_t B_pro
   return workspace_layout(N, D_in, D_out, B_proj, dt).total;
 }
 
+size_t rmm_workspace_bytes_for(int64_t N, int64_t D_in, int64_t D_out, int64_t B_proj, rmm_dtype dt, rmm_dist dist) {
+  const size_t base = rmm_workspace_bytes(N, D_in, D_out, B_proj, dt);
+  if (base == 0 || dist != RMM_DIST_SORS_HADAMARD || dt != RMM_DTYPE_BF16) return base;
+  const Workspace w = workspace_layout(N, D_in, D_out, B_proj, dt);
+  const size_t f = sors_fast_full_scratch(B_proj, D_in, N), b = sors_fast_full_scratch(B_proj, D_out, N);
+  const size_t want = w.scratch_off + (f > b ? f : b);
+  return want > base ? want : base;
+}
+
 rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, int64_t D_in, int64_t D_out,
                        uint64_t seed, int64_t B_proj, rmm_dist dist, rmm_dtype dt, void* Y, void* X_proj,
                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
@@ -819,7 +836,7 @@ rmm_status rmm_forward(const void* X, const void* W, const void* b, int64_t N, i
   if (dt == RMM_DTYPE_BF16) {
     float* scratch = reinterpret_cast<float*>(ws + w.scratch_off);
     unsigned long long* tickets = reinterpret_cast<unsigned long long*>(ws + w.ticket_off);
-    const size_t scratch_bytes = w.total - w.scratch_off;
+    const size_t scratch_bytes = workspace_bytes - w.scratch_off;   // all the caller gave: the fast Hadamard path uses the extra
     // the first kernel of the call resets the status word (no separate memset on the stream)
     if (dist == RMM_DIST_SORS_HADAMARD && sors_fast_supported(B_proj, D_in, N, scratch_bytes)) {
       // the subsampled-Hadamard sketch by its fast transform; the dense product on its own
@@ -891,7 +908,7 @@ rmm_status rmm_backward(const void* dY, const void* W, const void* X_proj, int64
   if (dt == RMM_DTYPE_BF16) {
     float* scratch = reinterpret_cast<float*>(ws + w.scratch_off);
     unsigned long long* tickets = reinterpret_cast<unsigned long long*>(ws + w.ticket_off);
-    const size_t scratch_bytes = w.total - w.scratch_off;
+    const size_t scratch_bytes = workspace_bytes - w.scratch_off;   // all the caller gave: the fast Hadamard path uses the extra
     // the first kernel of the call resets the status word (no separate memset on the stream)
     if (dist == RMM_DIST_SORS_HADAMARD && sors_fast_supported(B_proj, D_out, N, scratch_bytes)) {
       if (dX) {

@@ -28,8 +28,9 @@ class Workspace:
     def __init__(self):
         self.buf = None
 
-    def get(self, N, D_in, D_out, B_proj, dt, device):
-        need = P.rmm_workspace_bytes(N, D_in, D_out, B_proj, dt)
+    def get(self, N, D_in, D_out, B_proj, dt, device, dist=None):
+        need = P.rmm_workspace_bytes(N, D_in, D_out, B_proj, dt) if dist is None else \
+            P.rmm_workspace_bytes_for(N, D_in, D_out, B_proj, dt, dist)
         if self.buf is None or self.buf.numel() < need or self.buf.device != device:
             self.buf = torch.empty(need, dtype=torch.uint8, device=device)
         return self.buf
@@ -48,7 +49,7 @@ class RMMLinearFunction(torch.autograd.Function):
             x2 = x2.contiguous()
         n = x2.shape[0]
         dt = P.RMM_DTYPE_BF16 if x.dtype == torch.bfloat16 else P.RMM_DTYPE_F32
-        ws = workspace.get(n, d_in, weight.shape[0], b_proj, dt, x.device)
+        ws = workspace.get(n, d_in, weight.shape[0], b_proj, dt, x.device, dist)
         y, x_proj = P.rmm_forward(x2, weight, bias, seed, b_proj, dist, workspace=ws)
         ctx.save_for_backward(weight, x_proj)
         ctx.rmm = (seed, dist, x.shape, bias is not None, workspace, trace)
@@ -69,7 +70,7 @@ class RMMLinearFunction(torch.autograd.Function):
             dy2 = dy2.contiguous()
         n = dy2.shape[0]
         dt = P.RMM_DTYPE_BF16 if dy.dtype == torch.bfloat16 else P.RMM_DTYPE_F32
-        ws = workspace.get(n, d_in, d_out, x_proj.shape[0], dt, dy.device)
+        ws = workspace.get(n, d_in, d_out, x_proj.shape[0], dt, dy.device, dist)
         want_dx = ctx.needs_input_grad[0]
         dx, dw, db = P.rmm_backward(dy2, weight, x_proj, seed, dist, workspace=ws, want_dx=want_dx, want_db=has_bias)
         if trace is not None:

@@ -57,6 +57,28 @@ def test_workspace_bytes(lib):
     assert f(0, 8, 8, 1, 0) == 0 and f(8, 8, 8, 9, 0) == 0 and f(8, 8, 8, 1, 7) == 0
 
 
+def test_workspace_bytes_for_a_sketch(lib):
+    """The suggested size is the smallest valid one except for the subsampled-Hadamard sketch in bf16 mode inside the fast
+    path's range (Hadamard order 128 .. 16384), where it adds room for the transform's intermediate: L x D bf16 values."""
+    base = lib.rmm_workspace_bytes
+    base.restype = C.c_size_t
+    base.argtypes = [C.c_int64] * 4 + [C.c_int]
+    f = lib.rmm_workspace_bytes_for
+    f.restype = C.c_size_t
+    f.argtypes = [C.c_int64] * 4 + [C.c_int, C.c_int]
+    shape = (16384, 1024, 4096, 1638)
+    small = base(*shape, 0)
+    for dist in (0, 1, 2, 4):
+        assert f(*shape, 0, dist) == small
+    roomy = f(*shape, 0, 3)
+    assert roomy % 256 == 0 and roomy >= small and roomy >= 16384 * 4096 * 2       # T for all of dY's columns
+    assert roomy < small + 16384 * 4096 * 2 + (16 << 20)
+    assert f(*shape, 1, 3) == base(*shape, 1)                                      # fp32 mode: no fast path
+    assert f(16500, 1024, 4096, 1638, 0, 3) == base(16500, 1024, 4096, 1638, 0)    # Hadamard order 32768: dense kernel
+    assert f(100, 64, 64, 10, 0, 3) == base(100, 64, 64, 10, 0)                    # the smallest size already has room
+    assert f(0, 8, 8, 1, 0, 3) == 0 and f(8, 8, 8, 9, 0, 3) == 0
+
+
 def test_argument_errors_are_reported_before_any_launch(lib):
     i64, vp = C.c_int64, C.c_void_p
     fwd = lib.rmm_forward

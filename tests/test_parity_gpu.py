@@ -301,7 +301,7 @@ def test_host_buffer_entry_points():
 
 
 # ------------------------------------------------------------------ full-size workloads, sampled outputs
-def _sampled_full_size(name):
+def _sampled_full_size(name, roomy=False):
     """The launch configuration the benchmark times, checked on outputs the oracle computes one by one: one row
     of Y and of dX in every 128-row block (every row block of every output tile), one row of X_proj in every
     128-row sketch tile plus the first and last, one row of dW in every 128-row block, all of db; all columns of
@@ -313,7 +313,8 @@ def _sampled_full_size(name):
     X, W, b, dY = R.make_inputs(w)
     N, k, Di, Do = w.n_tokens, w.b_proj, w.d_in, w.d_out
     Xd, Wd, dYd = to_dev(X, w.dtype), to_dev(W, w.dtype), to_dev(dY, w.dtype)
-    ws = P.alloc_workspace(N, Di, Do, k, w.dtype)
+    # roomy: the workspace size the library suggests for this sketch (what the benchmark allocates) instead of the smallest
+    ws = P.alloc_workspace(N, Di, Do, k, w.dtype, dist=w.dist if roomy else None)
     Y, Xp = P.rmm_forward(Xd, Wd, None, w.seed, k, w.dist, workspace=ws)
     dX, dW, db = P.rmm_backward(dYd, Wd, Xp, w.seed, w.dist, workspace=ws)
     torch.cuda.synchronize()
@@ -366,6 +367,18 @@ def _sampled_full_size(name):
                                   "large_ffn_up_sors_rho0.1", "large_ffn_up_dct_rho0.1"])
 def test_full_size_sampled(name):
     assert _sampled_full_size(name)
+
+
+def test_full_size_sampled_suggested_workspace():
+    """The subsampled-Hadamard fast path with the workspace of rmm_workspace_bytes_for: all of dY's columns in one round
+    (with the smallest workspace, above, it takes them in two)."""
+    P = _P()
+    w = R.WORKLOADS["large_ffn_up_sors_rho0.1"]
+    small = P.rmm_workspace_bytes(w.n_tokens, w.d_in, w.d_out, w.b_proj, w.dtype)
+    roomy = P.rmm_workspace_bytes_for(w.n_tokens, w.d_in, w.d_out, w.b_proj, w.dtype, w.dist)
+    assert roomy > small
+    assert P.rmm_workspace_bytes_for(w.n_tokens, w.d_in, w.d_out, w.b_proj, w.dtype, R.DIST_GAUSSIAN) == small
+    assert _sampled_full_size("large_ffn_up_sors_rho0.1", roomy=True)
 
 
 @pytest.mark.parametrize("name", ["base_ffn_up_rho0.1", "base_ffn_up_rho0.5", "base_ffn_up_rho0.9"])
