@@ -210,6 +210,15 @@ int64_t rmm_debug_pass_schedule(int64_t gemm_m, int64_t gemm_n, int64_t gemm_k, 
                                 int64_t tokens, int max_pairs, int64_t* out, int64_t cap);
 
 /*
+ * Host-only testing aid (no device needed): how the fast transform of RMM_DIST_SORS_HADAMARD (bf16 mode) would
+ * take a sketch of `rows` rows over a tokens x cols matrix with `scratch_bytes` bytes of scratch (the part of the
+ * workspace that follows the status word, the flags and G).
+ * Returns 1 and writes info[0..3] = Hadamard order L, L / 128, columns per round, rounds (two launches each);
+ * 0 when the shape is outside the fast path (the dense sketch kernel is used); -1 for invalid arguments.
+ */
+int rmm_debug_hadamard_plan(int64_t rows, int64_t cols, int64_t tokens, size_t scratch_bytes, int64_t* info);
+
+/*
  * Reads the status word that the kernels of the last call using this workspace left
  * there.  HOST-synchronous on the device-to-host copy of one word: the caller must
  * have synchronised the stream first.  Returns RMM_OK or RMM_ERR_TIMEOUT (or

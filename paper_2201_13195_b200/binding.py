@@ -22,7 +22,7 @@ EXPORTS = ("rmm_workspace_bytes", "rmm_workspace_bytes_for", "rmm_forward", "rmm
            "rmm_last_device_status", "rmm_status_string", "rmm_host_staging_bytes",
            "rmm_forward_host", "rmm_backward_host", "rmm_profile_enable", "rmm_profile_read",
            "rmm_bias_grad_static", "rmm_debug_gauss_words", "rmm_debug_sketch_schedule",
-           "rmm_variance_probe_workspace_bytes", "rmm_variance_probe", "rmm_debug_pass_schedule", "rmm_layer_launch_count", "rmm_set_pass_mode")
+           "rmm_variance_probe_workspace_bytes", "rmm_variance_probe", "rmm_debug_pass_schedule", "rmm_debug_hadamard_plan", "rmm_layer_launch_count", "rmm_set_pass_mode")
 RMM_BIAS_GRAD_STATIC_MAX_D_OUT = 4096
 STEP_NAMES = ("y", "sketch", "dx", "sdy", "dw", "db", "fwd", "bwd")
 
@@ -60,6 +60,8 @@ _lib.rmm_debug_sketch_schedule.argtypes = [_i64, _i64, _i64, _int, _int, _vp, _i
 _lib.rmm_debug_sketch_schedule.restype = _i64
 _lib.rmm_debug_pass_schedule.argtypes = [_i64, _i64, _i64, _i64, _i64, _i64, _int, _vp, _i64]
 _lib.rmm_debug_pass_schedule.restype = _i64
+_lib.rmm_debug_hadamard_plan.argtypes = [_i64, _i64, _i64, _sz, C.POINTER(C.c_int64)]
+_lib.rmm_debug_hadamard_plan.restype = _int
 _lib.rmm_variance_probe_workspace_bytes.argtypes = [_i64, _i64, _i64]
 _lib.rmm_variance_probe_workspace_bytes.restype = _sz
 _lib.rmm_variance_probe.argtypes = [_vp, _vp, _i64, _i64, _i64, _i64, _int, _int, _vp, _vp, _vp, _sz, _vp]
@@ -286,6 +288,17 @@ def rmm_debug_pass_trace():
 
 def rmm_layer_launch_count() -> int:
     return int(_lib.rmm_layer_launch_count())
+
+
+def rmm_debug_hadamard_plan(rows, cols, tokens, scratch_bytes):
+    """How the fast Hadamard transform would take a sketch (host only): dict, or None outside the fast path."""
+    info = (C.c_int64 * 4)()
+    r = _lib.rmm_debug_hadamard_plan(rows, cols, tokens, scratch_bytes, info)
+    if r < 0:
+        raise ValueError("invalid arguments")
+    if r == 0:
+        return None
+    return {"order": int(info[0]), "blocks": int(info[1]), "columns_per_round": int(info[2]), "rounds": int(info[3])}
 
 
 def rmm_debug_pass_schedule(gemm, sketch, max_pairs=74):

@@ -1049,6 +1049,17 @@ int64_t rmm_debug_sketch_schedule(int64_t rows, int64_t cols, int64_t tokens, in
   return n;
 }
 
+int rmm_debug_hadamard_plan(int64_t rows, int64_t cols, int64_t tokens, size_t scratch_bytes, int64_t* info) {
+  if (rows < 1 || cols < 1 || tokens < 1 || info == nullptr) return -1;
+  SorsFastPlan plan;
+  if (!sors_fast_plan(rows, cols, tokens, scratch_bytes, &plan)) return 0;
+  info[0] = (int64_t)plan.mask + 1;
+  info[1] = plan.A;
+  info[2] = plan.wslab;
+  info[3] = (cols + plan.wslab - 1) / plan.wslab;
+  return 1;
+}
+
 int64_t rmm_debug_pass_schedule(int64_t gemm_m, int64_t gemm_n, int64_t gemm_k, int64_t rows, int64_t cols, int64_t tokens,
                                 int max_pairs, int64_t* out, int64_t cap) {
   if (max_pairs < 1 || gemm_m < 0 || rows < 0) return -1;

@@ -79,6 +79,26 @@ def test_workspace_bytes_for_a_sketch(lib):
     assert f(0, 8, 8, 1, 0, 3) == 0 and f(8, 8, 8, 9, 0, 3) == 0
 
 
+def test_hadamard_fast_path_plan(lib):
+    """Rounds of the fast transform: the intermediate T (L x columns, bf16) has to fit the scratch it is given."""
+    f = lib.rmm_debug_hadamard_plan
+    f.restype = C.c_int
+    f.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_size_t, C.POINTER(C.c_int64)]
+    info = (C.c_int64 * 4)()
+    mib = 1 << 20
+    assert f(1639, 4096, 16384, 160 * mib, info) == 1
+    assert list(info) == [16384, 128, 4096, 1]                      # all of dY's columns at once
+    assert f(1639, 4096, 16384, 70 * mib, info) == 1
+    assert info[3] == 2 and info[2] == 2048 and info[2] % 64 == 0   # two equal rounds rather than a full and a narrow one
+    assert f(1639, 4096, 16384, 40 * mib, info) == 1 and info[3] == 4 and info[2] == 1024
+    assert f(77, 520, 389, 8 * mib, info) == 1 and list(info) == [512, 4, 576, 1]     # ragged width: whole 64-column slabs
+    assert f(128, 72, 128, 8 * mib, info) == 1 and info[0] == 128 and info[1] == 1
+    assert f(5, 40, 37, 8 * mib, info) == 0                         # Hadamard order 64: dense kernel
+    assert f(141, 1024, 16500, 512 * mib, info) == 0                # order 32768: dense kernel
+    assert f(1639, 4096, 16384, 1 * mib, info) == 0                 # not even one slab of T fits
+    assert f(0, 8, 8, mib, info) == -1 and f(8, 8, 8, mib, None) == -1
+
+
 def test_argument_errors_are_reported_before_any_launch(lib):
     i64, vp = C.c_int64, C.c_void_p
     fwd = lib.rmm_forward
