@@ -299,14 +299,20 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    t_warm = time.perf_counter()
     for i in range(args.warmup):
         step(i)
     barrier()
+    t_warm = (time.perf_counter() - t_warm) / max(args.warmup, 1)
     assert P.rmm_last_device_status(ws) == P.RMM_OK
 
     launches_before = P.rmm_layer_launch_count()
-    P.rmm_profile_enable(min(args.steps, 200) * 6)     # per-kernel events for the first 200 timed steps
-    sampler = ClockSampler(physical_gpu_index(local_rank))
+    # per-kernel events for the first 50 timed steps only: a pair of events per pass costs a 4096-token step 6 %
+    P.rmm_profile_enable(min(args.steps, 50) * 6)
+    # about fifty samples over the timed region, at least one per millisecond's worth of it for short runs: a sampler
+    # thread that wakes every millisecond competes with the launching thread of a host-bound (4096-token) run
+    period = min(0.05, max(0.001, t_warm * args.steps / 50))
+    sampler = ClockSampler(physical_gpu_index(local_rank), period)
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -320,7 +326,7 @@ def main():
     gpu_launches = P.rmm_layer_launch_count() - launches_before     # the library's own count of its kernel launches
     ms_total = e0.elapsed_time(e1)
     assert P.rmm_last_device_status(ws) == P.RMM_OK
-    records = P.rmm_profile_read(min(args.steps, 200) * 6)
+    records = P.rmm_profile_read(min(args.steps, 50) * 6)
     P.rmm_profile_enable(0)
     if args.cycle_trace and rank == 0:
         tr = P.rmm_debug_pass_trace()
